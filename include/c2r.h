@@ -1,0 +1,277 @@
+/*
+ * c2r.h -- C ABI of the B200 (sm_100a) hot path of collaboration-constrained routing (C2R)
+ * for Mixture-of-Experts layers (arXiv 2504.01337).
+ *
+ * Conventions, valid for every call unless its comment says otherwise
+ *   - Pointers are DEVICE pointers; the few host pointers are named *_host.
+ *   - The caller owns every buffer.  The library allocates no device memory, keeps no pointer
+ *     after the enqueued kernels finish, never synchronises the stream and never traps.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - Return value: C2R_OK or a negative c2r_error.  Argument and shape checks run on the host
+ *     before anything is enqueued; after C2R_ERR_CUDA, c2r_last_cuda_error() gives the
+ *     cudaError_t of the failed runtime call.
+ *   - Matrices are row-major and dense.  "T" below is the storage type selected by
+ *     cfg->dtype: float (C2R_F32) or bfloat16 (C2R_BF16).  Accumulation is always fp32.
+ *     The per-(token, expert) partial results that are summed over k afterwards (Yp, Ys, dXp,
+ *     dXs) are always float, so that the only rounding to T on the output path is the final one.
+ *   - Notation follows the paper: N tokens, d hidden size, E routed experts, I expert
+ *     intermediate size, K experts per token, T collaborator-set size, P logical partitions.
+ *   - Shape limits: 1 <= K <= 8, K-1 <= T <= E-1, E <= 64 (E <= 63 with a shared expert),
+ *     d % 8 == 0, I % 16 == 0, 1 <= P <= E, N*K < 2^30.
+ */
+#ifndef C2R_H_
+#define C2R_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum c2r_error {
+  C2R_OK = 0,
+  C2R_ERR_INVALID_ARG = -1,       /* NULL where a buffer is required, or a value out of range */
+  C2R_ERR_UNSUPPORTED_SHAPE = -2, /* a documented shape limit is violated */
+  C2R_ERR_WORKSPACE = -3,         /* workspace missing or smaller than c2r_workspace_bytes() */
+  C2R_ERR_CUDA = -4               /* a CUDA runtime / driver call failed */
+} c2r_error;
+
+enum { C2R_F32 = 0, C2R_BF16 = 1 };
+
+/* status bits OR-ed into the optional device status word of c2r_route / c2r_permute */
+enum {
+  C2R_STATUS_NAN_LOGIT = 1,     /* a NaN logit was ordered as -inf */
+  C2R_STATUS_SET_TOO_SMALL = 2, /* a collaborator mask offered fewer than K-1 experts */
+  C2R_STATUS_BAD_INDEX = 4,     /* an expert index outside [0,E) was clamped */
+  C2R_STATUS_WAIT_TIMEOUT = 8   /* a bounded wait inside a kernel gave up */
+};
+
+typedef struct c2r_config {
+  int32_t N;         /* tokens in the batch */
+  int32_t d;         /* hidden size */
+  int32_t E;         /* routed experts */
+  int32_t I;         /* intermediate size of a routed expert */
+  int32_t K;         /* experts per token */
+  int32_t T;         /* collaborator-set size, |Top-T(E_i)| (Eq. 4) */
+  int32_t P;         /* logical expert partitions (expert-parallel degree that is modelled) */
+  int32_t I_s;       /* intermediate size of the always-on shared expert, 0 = none */
+  int32_t dtype;     /* C2R_F32 or C2R_BF16 */
+  int32_t row_align; /* every expert's segment of the permuted layout starts at a multiple of this
+                        (>= 1; the tensor-core GEMMs of the bf16 path need a multiple of 128) */
+  int32_t renorm;    /* 1: weights = softmax over the K kept logits (Eq. 1); 0: full-softmax probabilities */
+  int32_t flags;     /* reserved, 0 */
+} c2r_config;
+
+enum { C2R_WS_PERMUTE = 0, C2R_WS_GATE_BWD = 1, C2R_WS_LAYER = 2 };
+
+/* Bytes of scratch the named call needs for this configuration (host function). */
+size_t c2r_workspace_bytes(const c2r_config* cfg, int which);
+
+/* Rows the permuted buffers (Xp, Yp, ...) must hold: N*K plus worst-case alignment padding. */
+int64_t c2r_permuted_rows(const c2r_config* cfg);
+
+/* cudaError_t of the last failed CUDA call made by this library on the calling thread. */
+int c2r_last_cuda_error(void);
+
+/* Sec. 3.1, Eq. 1 (argument of Top-K): L[t,e] = <X[t,:], Wg[e,:]>.
+ * X [N,d] T; Wg [E,d] T; wsg [d] T or NULL (gate vector of the shared expert);
+ * out: L [N,E] float; z [N] float = <X[t,:], wsg> (required iff wsg != NULL). */
+int c2r_gate_logits(const c2r_config* cfg, const void* X, const void* Wg, const void* wsg,
+                    float* L, float* z, void* stream);
+
+/* Sec. 3.3 step 2 (C2R) and Eq. 1 (conventional Top-K when mask == NULL).
+ * The top-1 expert i* is the arg-max of L[t,:]; the other K-1 experts are the best-scoring
+ * j with bit j of mask[i*] set.  Order everywhere: (logit descending, index ascending);
+ * NaN orders as -inf.  Selection is made on the raw fp32 logits.
+ * L [N,E] float; mask [E] uint64 or NULL;
+ * out: idx [N,K] int32 (column 0 = top-1, then selection order); w [N,K] float (Eq. 1 weights);
+ *      p [N,E] float full-row softmax or NULL; status: one int32 (OR of C2R_STATUS_*) or NULL. */
+int c2r_route(const c2r_config* cfg, const float* L, const uint64_t* mask, int32_t* idx, float* w,
+              float* p, int32_t* status, void* stream);
+
+/* Sec. 3.2, Eq. 2: C[i,j] = number of tokens whose selected set contains both i and j.
+ * idx [n_tokens,K] int32; C [E,E] int32.  accumulate != 0 adds to C (profiling over several
+ * batches), otherwise C is overwritten. */
+int c2r_collab_count(const c2r_config* cfg, const int32_t* idx, int64_t n_tokens, int32_t* C,
+                     int accumulate, void* stream);
+
+/* Sec. 3.3 step 1, Eq. 4: I_T[i,:] = the cfg->T experts j != i with the largest C[i,j]
+ * (ties: lower j); mask[i] has exactly those bits set.  C [E,E] int32; I_T [E,T] int32; mask [E] uint64. */
+int c2r_collab_sets(const c2r_config* cfg, const int32_t* C, int32_t* I_T, uint64_t* mask, void* stream);
+
+/* Sec. 3.4 (co-locate closely collaborating experts on one device).  HOST function, host arrays.
+ * mode 0 (greedy): partition p holds floor(E/P) + (p < E mod P) experts; it is seeded with the
+ * unassigned expert of largest C[e,e] and grown by the unassigned expert with the largest summed
+ * co-activation with its members (ties: lower id).  mode 1: part[e] = floor(e*P/E).
+ * out: part_host [E]; rank_host [E] = position of expert e in the partition-major,
+ * id-ascending layout order. */
+int c2r_place_experts(const c2r_config* cfg, const int32_t* C_host, int mode, int32_t* part_host,
+                      int32_t* rank_host);
+
+/* The "dispatch" of Sec. 3.1 on one device: stable counting sort of the slots s = t*K+k by
+ * expert_rank[idx[s]] (NULL = identity), then the row gather.
+ * out: counts [E] int32; offsets [E+1] int32 (start row of expert e, a multiple of row_align;
+ * offsets[E] = end of the layout); row_of_slot [N*K] int32; slot_of_row [c2r_permuted_rows] int32
+ * (-1 = padding); Xp [c2r_permuted_rows, d] T with Xp[r,:] = X[slot_of_row[r]/K,:], padding rows zero.
+ * X == NULL builds the index only.  Atomic-free and deterministic.
+ * ws: C2R_WS_PERMUTE bytes.  status as in c2r_route. */
+int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
+                int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp,
+                int32_t* status, void* ws, size_t ws_bytes, void* stream);
+
+/* Weight layout used by the fused SwiGLU kernels (no counterpart in the paper).
+ * W1 (gate projection) and W3 (up projection), both [n_experts, I, d] T, are interleaved in
+ * blocks of 128 intermediate channels: block j holds rows [128j, 128j+b) of W1 followed by the
+ * same rows of W3, b = min(128, I-128j).  W13p [n_experts, 2I, d] T.  unpack is the inverse and
+ * also converts a gradient in packed layout back to (dW1, dW3). */
+int c2r_pack_weights(const c2r_config* cfg, int n_experts, int I, const void* W1, const void* W3,
+                     void* W13p, void* stream);
+int c2r_unpack_weights(const c2r_config* cfg, int n_experts, int I, const void* W13p, void* W1,
+                       void* W3, void* stream);
+
+/* Sec. 3.1 ("each token is fed to its selected experts"), expert = SwiGLU MLP without biases.
+ * For each expert e on rows [offsets[e], offsets[e]+counts[e]) of Xp:
+ *   A = Xp W1_e^T, B = Xp W3_e^T, H = silu(A) * B, Yp = H W2_e^T.
+ * Xp [R,d] T; counts [n_experts], offsets [n_experts+1] int32 (device); W13p packed (above);
+ * W2 [n_experts, d, I] T.  out: AB [R, 2I] T (A and B in the packed column layout, kept for the
+ * backward pass), H [R,I] T, Yp [R,d] float.
+ * R = rows of the buffers.  Padding rows of Xp must be zero.  n_experts = 1 with counts = {R},
+ * offsets = {0,R} evaluates the dense shared expert. */
+int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
+                           const int32_t* counts, const int32_t* offsets, const void* W13p,
+                           const void* W2, void* AB, void* H, void* Yp, void* stream);
+
+/* Backward of the above:  dH = dYp W2; dA = dH * B * silu'(A); dB = dH * silu(A);
+ * dXp = dA W1 + dB W3; dW2_e = dYp^T H; dW1_e = dA^T Xp; dW3_e = dB^T Xp.
+ * dYp [R,d] T (padding rows zero); out: dAB [R,2I] T (packed columns), dXp [R,d] float,
+ * dW13p [n_experts,2I,d] T (packed rows), dW2 [n_experts,d,I] T.  accumulate != 0 adds into the
+ * weight gradients. */
+int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
+                           const int32_t* counts, const int32_t* offsets, const void* W13p,
+                           const void* W2, const void* AB, const void* H, const void* dYp, void* dAB,
+                           void* dXp, void* dW13p, void* dW2, int accumulate, void* stream);
+
+/* Sec. 3.1 (weighted sum of the selected experts' outputs):
+ * Y[t,:] = sum_k w[t,k] * Yp[row_of_slot[t*K+k],:]  (k ascending, fp32)
+ *          + sigmoid(z[t]) * Ys[t,:] when Ys != NULL (gated shared expert).
+ * Yp [R,d] float; Ys [N,d] float; out: Y [N,d] T. */
+int c2r_combine(const c2r_config* cfg, const void* Yp, const float* w, const int32_t* row_of_slot,
+                const void* Ys, const float* z, void* Y, void* stream);
+
+/* Backward of c2r_combine: dYp[row(t,k),:] = w[t,k] dY[t,:] (padding rows zeroed);
+ * dw[t,k] = <dY[t,:], Yp[row(t,k),:]>; dYs = sigmoid(z) dY; dz = <dY,Ys> sigmoid'(z).
+ * dY [N,d] T; Yp, Ys float; out: dYp [R,d] T; dYs [N,d] T; dw [N,K], dz [N] float. */
+int c2r_combine_bwd(const c2r_config* cfg, const void* dY, const void* Yp, const float* w,
+                    const int32_t* row_of_slot, const int32_t* slot_of_row, const void* Ys, const float* z,
+                    void* dYp, float* dw, void* dYs, float* dz, void* stream);
+
+/* Backward of Eq. 1's softmax over the kept logits (cfg->renorm must be 1):
+ * dl[t,k] = w[t,k] (dw[t,k] - sum_j w[t,j] dw[t,j]) -- the gradient w.r.t. L[t, idx[t,k]];
+ * all other entries of dL are zero. */
+int c2r_route_bwd(const c2r_config* cfg, const float* w, const float* dw, float* dl, void* stream);
+
+/* Gate weight gradients: dWg[e,:] = sum_t dL[t,e] X[t,:], evaluated over expert e's rows of Xp
+ * (dl addressed through slot_of_row); dwsg[:] = sum_t dz[t] X[t,:].
+ * out: dWg [E,d] float; dwsg [d] float (iff dz != NULL).  ws: C2R_WS_GATE_BWD bytes. */
+int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
+                 const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
+                 float* dWg, float* dwsg, void* ws, size_t ws_bytes, void* stream);
+
+/* Gradient w.r.t. the hidden states (transpose of the dispatch, done as an atomic-free gather-sum):
+ * dX[t,:] = sum_k dXp[row_of_slot[t*K+k],:]  + dXs[t,:]                (shared expert, optional)
+ *           + sum_k dl[t,k] Wg[idx[t,k],:] + dz[t] wsg[:]              (gate, optional)
+ *           + dX[t,:] when accumulate != 0.
+ * dXp [R,d] float; dXs [N,d] float; out: dX [N,d] T. */
+int c2r_unpermute_grad(const c2r_config* cfg, const void* dXp, const int32_t* row_of_slot, const void* dXs,
+                       const int32_t* idx, const float* dl, const void* Wg, const float* dz, const void* wsg,
+                       void* dX, int accumulate, void* stream);
+
+/* Sec. 3.4 / Sec. 4.1 (token redundancy of the all-to-all).  part [E] int32 maps expert -> partition,
+ * home(t) = floor(t*P/N).  out (device, overwritten):
+ *   totals[0] = naive   = N*K rows (one per (token, expert));
+ *   totals[1] = dedup   = number of distinct (token, partition) pairs (zero-redundancy scheme);
+ *   totals[2], totals[3] = the same two counting only destinations != home(t);
+ *   send_naive, send_dedup [P,P] uint64: rows from home partition src to partition dst.
+ * redundancy r = 1 - dedup/naive. */
+int c2r_dispatch_volume(const c2r_config* cfg, const int32_t* idx, const int32_t* part, uint64_t* totals,
+                        uint64_t* send_naive, uint64_t* send_dedup, void* stream);
+
+/* Buffers of one layer for the drivers below.  Unused members may be NULL (no shared expert:
+ * every *s member; inference: every backward member). */
+typedef struct c2r_layer_buffers {
+  /* inputs and parameters */
+  const void* X;              /* [N,d] T */
+  const void* Wg;             /* [E,d] T */
+  const void* wsg;            /* [d] T */
+  const void* W13p;           /* [E,2I,d] T packed */
+  const void* W2;             /* [E,d,I] T */
+  const void* Ws13p;          /* [1,2I_s,d] T packed */
+  const void* Ws2;            /* [1,d,I_s] T */
+  const uint64_t* mask;       /* [E] collaborator masks, NULL = conventional Top-K */
+  const int32_t* expert_rank; /* [E] or NULL */
+  const int32_t* part;        /* [E] or NULL (dispatch volume skipped) */
+  /* forward state */
+  float* L;             /* [N,E] */
+  float* z;             /* [N] */
+  int32_t* idx;         /* [N,K] */
+  float* w;             /* [N,K] */
+  int32_t* counts;      /* [E] */
+  int32_t* offsets;     /* [E+1] */
+  int32_t* row_of_slot; /* [N*K] */
+  int32_t* slot_of_row; /* [R] */
+  void* Xp;             /* [R,d] */
+  void* AB;             /* [R,2I] */
+  void* H;              /* [R,I] */
+  void* Yp;             /* [R,d] float */
+  void* ABs;            /* [N,2I_s] */
+  void* Hs;             /* [N,I_s] */
+  void* Ys;             /* [N,d] float */
+  int32_t* s_counts;    /* [1]  = {N}   (device) */
+  int32_t* s_offsets;   /* [2]  = {0,N} (device) */
+  void* Y;              /* [N,d] T: layer output */
+  uint64_t* volume;     /* [4 + 2*P*P] totals, send_naive, send_dedup */
+  int32_t* status;      /* one int32 */
+  /* backward */
+  const void* dY; /* [N,d] T */
+  void* dYp;      /* [R,d] */
+  void* dAB;      /* [R,2I] */
+  void* dXp;      /* [R,d] float */
+  void* dYs;      /* [N,d] */
+  void* dABs;     /* [N,2I_s] */
+  void* dXs;      /* [N,d] float */
+  float* dw;      /* [N,K] */
+  float* dl;      /* [N,K] */
+  float* dz;      /* [N] */
+  void* dW13p;    /* [E,2I,d] T */
+  void* dW2;      /* [E,d,I] T */
+  void* dWs13p;   /* [1,2I_s,d] T */
+  void* dWs2;     /* [1,d,I_s] T */
+  float* dWg;     /* [E,d] */
+  float* dwsg;    /* [d] */
+  void* dX;       /* [N,d] T */
+  /* live profiling (c2r_train_step) */
+  int32_t* C;          /* [E,E] */
+  int32_t* I_T;        /* [E,T] */
+  uint64_t* mask_next; /* [E]: sets for the next step */
+  /* scratch */
+  void* ws;        /* C2R_WS_LAYER bytes */
+  size_t ws_bytes;
+} c2r_layer_buffers;
+
+/* Forward of the whole layer on one stream, no host synchronisation:
+ * gate -> route (C2R or Top-K) -> permute -> grouped SwiGLU (+ shared expert) -> combine
+ * (-> dispatch volume when part != NULL). */
+int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, void* stream);
+
+/* Backward of c2r_layer_fwd (routing decision frozen) using the state it left in `b`. */
+int c2r_layer_bwd(const c2r_config* cfg, const c2r_layer_buffers* b, int accumulate, void* stream);
+
+/* Forward, backward, then Eq. 2 and Eq. 4 on this step's routing: C is overwritten from idx and
+ * the refreshed sets are written to I_T / mask_next for the next step. */
+int c2r_train_step(const c2r_config* cfg, const c2r_layer_buffers* b, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* C2R_H_ */

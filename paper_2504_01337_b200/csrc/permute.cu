@@ -1,0 +1,610 @@
+// Dispatch on one device: atomic-free histogram / prefix-scan / stable rank over experts, the
+// 16-byte vectorised row gather, the weighted combine and their backward twins.
+#include "c2r_common.cuh"
+
+namespace c2r {
+
+constexpr int PERM_WARPS = 8;                 // warps per block
+constexpr int PERM_ITERS = 2;                 // 32-slot iterations per warp
+constexpr int PERM_BLOCK_SLOTS = PERM_WARPS * PERM_ITERS * 32;
+
+__device__ __forceinline__ uint32_t lanemask_lt() {
+  uint32_t m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+// Per-warp, per-expert counts of this block's slots.  A warp owns PERM_ITERS*32 consecutive
+// slots; inside a 32-slot group, lanes with equal expert form a peer set (match.any) whose
+// lowest lane adds the set size -- no atomics, and the order of slots is preserved.
+__device__ __forceinline__ void warp_count(const int32_t* __restrict__ idx, long long NK, int E, int (*warp_cnt)[64],
+                                           int e_reg[PERM_ITERS], int& flags) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const long long base = (long long)blockIdx.x * PERM_BLOCK_SLOTS + (long long)w * PERM_ITERS * 32;
+#pragma unroll
+  for (int it = 0; it < PERM_ITERS; ++it) {
+    const long long s = base + it * 32 + lane;
+    int e = -1;
+    if (s < NK) {
+      e = idx[s];
+      if (e < 0 || e >= E) { flags |= C2R_STATUS_BAD_INDEX; e = min(max(e, 0), E - 1); }
+    }
+    e_reg[it] = e;
+    const uint32_t peers = __match_any_sync(0xffffffffu, e);
+    if (e >= 0 && lane == __ffs(peers) - 1) warp_cnt[w][e] += __popc(peers);
+    __syncwarp();
+  }
+}
+
+__global__ void __launch_bounds__(PERM_WARPS * 32) perm_hist_kernel(const int32_t* __restrict__ idx, long long NK, int E,
+                                                                    int32_t* __restrict__ block_counts,
+                                                                    int32_t* __restrict__ status) {
+  __shared__ int warp_cnt[PERM_WARPS][64];
+  for (int i = threadIdx.x; i < PERM_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
+  __syncthreads();
+  int e_reg[PERM_ITERS];
+  int flags = 0;
+  warp_count(idx, NK, E, warp_cnt, e_reg, flags);
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    int s = 0;
+#pragma unroll
+    for (int w = 0; w < PERM_WARPS; ++w) s += warp_cnt[w][e];
+    block_counts[(size_t)blockIdx.x * E + e] = s;
+  }
+  if (status != nullptr && flags) atomicOr(status, flags);
+}
+
+// One block: per expert an exclusive scan of the block counts over blocks (a warp per expert,
+// 32 blocks per shuffle scan), then the segment offsets in layout (rank) order with alignment.
+__global__ void __launch_bounds__(1024) perm_scan_kernel(int32_t* __restrict__ block_counts, int n_blocks, int E,
+                                                         const int32_t* __restrict__ expert_rank, int row_align,
+                                                         int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+  __shared__ int s_counts[64];
+  __shared__ int s_by_rank[64];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int e = warp; e < E; e += 32) {
+    int running = 0;
+    for (int b0 = 0; b0 < n_blocks; b0 += 32) {
+      const int b = b0 + lane;
+      const int v = (b < n_blocks) ? block_counts[(size_t)b * E + e] : 0;
+      int incl = v;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        int o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+      }
+      if (b < n_blocks) block_counts[(size_t)b * E + e] = running + incl - v;
+      running += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) s_counts[e] = running;
+  }
+  if (threadIdx.x < E) {
+    int r = expert_rank ? expert_rank[threadIdx.x] : threadIdx.x;
+    r = min(max(r, 0), E - 1);
+    s_by_rank[r] = threadIdx.x;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int cursor = 0;
+    for (int r = 0; r < E; ++r) {
+      const int e = s_by_rank[r];
+      offsets[e] = cursor;
+      cursor += (s_counts[e] + row_align - 1) / row_align * row_align;
+    }
+    offsets[E] = cursor;
+  }
+  if (threadIdx.x < E) counts[threadIdx.x] = s_counts[threadIdx.x];
+}
+
+// Stable rank of every slot: segment start + slots of the same expert in earlier blocks, earlier
+// warps of this block, earlier 32-groups of this warp, lower lanes of this group.
+__global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_kernel(const int32_t* __restrict__ idx, long long NK, int E,
+                                                                    const int32_t* __restrict__ block_base,
+                                                                    const int32_t* __restrict__ offsets,
+                                                                    int32_t* __restrict__ row_of_slot,
+                                                                    int32_t* __restrict__ slot_of_row) {
+  __shared__ int warp_cnt[PERM_WARPS][64];
+  for (int i = threadIdx.x; i < PERM_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
+  __syncthreads();
+  int e_reg[PERM_ITERS];
+  int flags = 0;
+  warp_count(idx, NK, E, warp_cnt, e_reg, flags);
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    int run = offsets[e] + block_base[(size_t)blockIdx.x * E + e];
+#pragma unroll
+    for (int w = 0; w < PERM_WARPS; ++w) {
+      const int c = warp_cnt[w][e];
+      warp_cnt[w][e] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const long long base = (long long)blockIdx.x * PERM_BLOCK_SLOTS + (long long)w * PERM_ITERS * 32;
+#pragma unroll
+  for (int it = 0; it < PERM_ITERS; ++it) {
+    const long long s = base + it * 32 + lane;
+    const int e = e_reg[it];
+    const uint32_t peers = __match_any_sync(0xffffffffu, e);
+    const int start = (e >= 0) ? warp_cnt[w][e] : 0;
+    __syncwarp();
+    if (e >= 0 && lane == __ffs(peers) - 1) warp_cnt[w][e] = start + __popc(peers);
+    __syncwarp();
+    if (e >= 0) {
+      const int row = start + __popc(peers & lanemask_lt());
+      row_of_slot[s] = row;
+      slot_of_row[row] = (int32_t)s;
+    }
+  }
+}
+
+// Row gather, one warp per token: the token's row is read once and written to its K rows.
+template <typename T>
+__global__ void __launch_bounds__(256) permute_rows_kernel(const T* __restrict__ X,
+                                                           const int32_t* __restrict__ row_of_slot, T* __restrict__ Xp,
+                                                           int N, int d, int K) {
+  using V = Vec16<T>;
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= N) return;  // warp-uniform
+  const int my_row = (lane < K) ? row_of_slot[(size_t)t * K + lane] : 0;
+  int rows[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) rows[k] = __shfl_sync(0xffffffffu, my_row, k);
+  const int chunks = d / V::N;
+  const T* src = X + (size_t)t * d;
+  for (int c0 = lane; c0 < chunks; c0 += 32 * 4) {
+    V v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (c0 + 32 * u < chunks) v[u].load(src + (size_t)(c0 + 32 * u) * V::N);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (k >= K) break;
+      T* dst = Xp + (size_t)rows[k] * d;
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (c0 + 32 * u < chunks) v[u].store(dst + (size_t)(c0 + 32 * u) * V::N);
+    }
+  }
+}
+
+// Zero the padding rows (slot_of_row < 0) of a permuted buffer; one warp per row.
+template <typename T>
+__global__ void __launch_bounds__(256) zero_pad_rows_kernel(const int32_t* __restrict__ slot_of_row, T* __restrict__ Xp,
+                                                            long long R, int d) {
+  using V = Vec16<T>;
+  const int lane = threadIdx.x & 31;
+  const int chunks = d / V::N;
+  V zero;
+  float zf[V::N] = {};
+  zero.from_float(zf);
+  for (long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); r < R;
+       r += (long long)gridDim.x * (blockDim.x >> 5)) {
+    if (slot_of_row[r] >= 0) continue;
+    T* dst = Xp + (size_t)r * d;
+    for (int c = lane; c < chunks; c += 32) zero.store(dst + (size_t)c * V::N);
+  }
+}
+
+// Loads V::N consecutive elements of type S starting at p as floats (S = float or the storage type).
+template <typename T, typename S>
+__device__ __forceinline__ void load_as_float(const S* p, float* f) {
+  constexpr int NV = Vec16<T>::N;
+  if constexpr (sizeof(S) == 4) {
+#pragma unroll
+    for (int q = 0; q < NV / 4; ++q) {
+      const float4 v = *reinterpret_cast<const float4*>(p + 4 * q);
+      f[4 * q] = v.x; f[4 * q + 1] = v.y; f[4 * q + 2] = v.z; f[4 * q + 3] = v.w;
+    }
+  } else {
+    Vec16<S> v;
+    v.load(p);
+    v.to_float(f);
+  }
+}
+
+// out[t,:] = sum_k coef[t,k] * src[rows[t*K+k],:]            (coef == NULL -> 1)
+//          + ecoef(t) * extra[t,:]                           (ecoef = sigmoid(z[t]) if z else 1)
+//          + sum_k dl[t,k] * Wg[idx[t,k],:] + dz[t] * wsg[:] (gate terms, optional)
+//          + out[t,:] if accumulate.
+// src / extra are the fp32 partial results of the expert GEMMs; out has the storage type.
+// One warp per token, fp32 accumulation in k order.  Serves the combine and the gradient un-permute.
+template <typename T>
+__global__ void __launch_bounds__(256) gather_sum_kernel(const float* __restrict__ src, const int32_t* __restrict__ rows_g,
+                                                         const float* __restrict__ coef, const float* __restrict__ extra,
+                                                         const float* __restrict__ z, const int32_t* __restrict__ idx,
+                                                         const float* __restrict__ dl, const T* __restrict__ Wg,
+                                                         const float* __restrict__ dz, const T* __restrict__ wsg,
+                                                         T* __restrict__ out, int accumulate, int N, int d, int K) {
+  using V = Vec16<T>;
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= N) return;  // warp-uniform
+  int my_row = 0, my_idx = 0;
+  float my_coef = 1.f, my_dl = 0.f;
+  if (lane < K) {
+    my_row = rows_g[(size_t)t * K + lane];
+    if (coef) my_coef = coef[(size_t)t * K + lane];
+    if (dl) { my_dl = dl[(size_t)t * K + lane]; my_idx = idx[(size_t)t * K + lane]; }
+  }
+  int rows[8], eidx[8];
+  float cf[8], gl[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    rows[k] = __shfl_sync(0xffffffffu, my_row, k);
+    eidx[k] = __shfl_sync(0xffffffffu, my_idx, k);
+    cf[k] = __shfl_sync(0xffffffffu, my_coef, k);
+    gl[k] = __shfl_sync(0xffffffffu, my_dl, k);
+  }
+  const float ecoef = (extra && z) ? 1.0f / (1.0f + expf(-z[t])) : 1.0f;
+  const float dzt = (dz && wsg) ? dz[t] : 0.f;
+  const int chunks = d / V::N;
+  for (int c = lane; c < chunks; c += 32) {
+    const size_t col = (size_t)c * V::N;
+    float acc[V::N];
+#pragma unroll
+    for (int j = 0; j < V::N; ++j) acc[j] = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (k >= K) break;
+      float f[V::N];
+      load_as_float<T, float>(src + (size_t)rows[k] * d + col, f);
+#pragma unroll
+      for (int j = 0; j < V::N; ++j) acc[j] = fmaf(cf[k], f[j], acc[j]);
+    }
+    if (extra) {
+      float f[V::N];
+      load_as_float<T, float>(extra + (size_t)t * d + col, f);
+#pragma unroll
+      for (int j = 0; j < V::N; ++j) acc[j] = fmaf(ecoef, f[j], acc[j]);
+    }
+    if (dl) {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        if (k >= K) break;
+        float f[V::N];
+        load_as_float<T, T>(Wg + (size_t)eidx[k] * d + col, f);
+#pragma unroll
+        for (int j = 0; j < V::N; ++j) acc[j] = fmaf(gl[k], f[j], acc[j]);
+      }
+    }
+    if (dz && wsg) {
+      float f[V::N];
+      load_as_float<T, T>(wsg + col, f);
+#pragma unroll
+      for (int j = 0; j < V::N; ++j) acc[j] = fmaf(dzt, f[j], acc[j]);
+    }
+    T* o = out + (size_t)t * d + col;
+    if (accumulate) {
+      float f[V::N];
+      load_as_float<T, T>(o, f);
+#pragma unroll
+      for (int j = 0; j < V::N; ++j) acc[j] += f[j];
+    }
+    V r;
+    r.from_float(acc);
+    r.store(o);
+  }
+}
+
+// Backward of the combine, one warp per token.  Yp / Ys are the fp32 partials; dYp / dYs feed the
+// backward GEMMs and have the storage type.
+template <typename T>
+__global__ void __launch_bounds__(256) combine_bwd_kernel(const T* __restrict__ dY, const float* __restrict__ Yp,
+                                                          const float* __restrict__ w,
+                                                          const int32_t* __restrict__ rows_g,
+                                                          const float* __restrict__ Ys, const float* __restrict__ z,
+                                                          T* __restrict__ dYp, float* __restrict__ dw,
+                                                          T* __restrict__ dYs, float* __restrict__ dz, int N, int d,
+                                                          int K) {
+  using V = Vec16<T>;
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= N) return;  // warp-uniform
+  int my_row = 0;
+  float my_w = 0.f;
+  if (lane < K) { my_row = rows_g[(size_t)t * K + lane]; my_w = w[(size_t)t * K + lane]; }
+  int rows[8];
+  float wk[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    rows[k] = __shfl_sync(0xffffffffu, my_row, k);
+    wk[k] = __shfl_sync(0xffffffffu, my_w, k);
+  }
+  const float g = Ys ? 1.0f / (1.0f + expf(-z[t])) : 0.f;
+  float dot[9];
+#pragma unroll
+  for (int k = 0; k < 9; ++k) dot[k] = 0.f;
+  const int chunks = d / V::N;
+  for (int c = lane; c < chunks; c += 32) {
+    const size_t col = (size_t)c * V::N;
+    float gf[V::N];
+    load_as_float<T, T>(dY + (size_t)t * d + col, gf);
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (k >= K) break;
+      float yf[V::N], of[V::N];
+      load_as_float<T, float>(Yp + (size_t)rows[k] * d + col, yf);
+#pragma unroll
+      for (int j = 0; j < V::N; ++j) { dot[k] = fmaf(gf[j], yf[j], dot[k]); of[j] = wk[k] * gf[j]; }
+      V ov;
+      ov.from_float(of);
+      ov.store(dYp + (size_t)rows[k] * d + col);
+    }
+    if (Ys) {
+      float sf[V::N], of[V::N];
+      load_as_float<T, float>(Ys + (size_t)t * d + col, sf);
+#pragma unroll
+      for (int j = 0; j < V::N; ++j) { dot[8] = fmaf(gf[j], sf[j], dot[8]); of[j] = g * gf[j]; }
+      V ov;
+      ov.from_float(of);
+      ov.store(dYs + (size_t)t * d + col);
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < 9; ++k) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot[k] += __shfl_xor_sync(0xffffffffu, dot[k], off);
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (k < K) dw[(size_t)t * K + k] = dot[k];
+    if (Ys) dz[t] = dot[8] * g * (1.0f - g);
+  }
+}
+
+// dWg[e, cols] = sum over expert e's rows r of dl[slot_of_row[r]] * Xp[r, cols].
+// grid (d / (32*VEC), E); 8 warps split the rows, partial sums merged in warp order.
+template <typename T>
+__global__ void __launch_bounds__(256) gate_wgrad_kernel(const T* __restrict__ Xp, const int32_t* __restrict__ counts,
+                                                         const int32_t* __restrict__ offsets,
+                                                         const int32_t* __restrict__ slot_of_row,
+                                                         const float* __restrict__ dl, float* __restrict__ dWg, int d) {
+  using V = Vec16<T>;
+  __shared__ float part[8][32 * V::N];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int e = blockIdx.y;
+  const int col = (blockIdx.x * 32 + lane) * V::N;
+  const int r0 = offsets[e], r1 = r0 + counts[e];
+  float acc[V::N];
+#pragma unroll
+  for (int j = 0; j < V::N; ++j) acc[j] = 0.f;
+  if (col < d) {
+    for (int r = r0 + w; r < r1; r += 8) {
+      const float g = dl[slot_of_row[r]];
+      V v;
+      v.load(Xp + (size_t)r * d + col);
+      float f[V::N];
+      v.to_float(f);
+#pragma unroll
+      for (int j = 0; j < V::N; ++j) acc[j] = fmaf(g, f[j], acc[j]);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < V::N; ++j) part[w][lane * V::N + j] = acc[j];
+  __syncthreads();
+  for (int i = threadIdx.x; i < 32 * V::N; i += blockDim.x) {
+    float s = 0.f;
+#pragma unroll
+    for (int ww = 0; ww < 8; ++ww) s += part[ww][i];
+    const int c = blockIdx.x * 32 * V::N + i;
+    if (c < d) dWg[(size_t)e * d + c] = s;
+  }
+}
+
+// Partial column sums  ws[split, cols] = sum_{t in split} dz[t] * X[t, cols];  second kernel adds the splits in order.
+constexpr int GWS_SPLITS = 64;
+template <typename T>
+__global__ void __launch_bounds__(256) shared_gate_wgrad_kernel(const T* __restrict__ X, const float* __restrict__ dz,
+                                                                float* __restrict__ ws, int N, int d) {
+  using V = Vec16<T>;
+  __shared__ float part[8][32 * V::N];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int col = (blockIdx.x * 32 + lane) * V::N;
+  const int per = (N + GWS_SPLITS - 1) / GWS_SPLITS;
+  const int t0 = blockIdx.y * per, t1 = min(N, t0 + per);
+  float acc[V::N];
+#pragma unroll
+  for (int j = 0; j < V::N; ++j) acc[j] = 0.f;
+  if (col < d) {
+    for (int t = t0 + w; t < t1; t += 8) {
+      const float g = dz[t];
+      V v;
+      v.load(X + (size_t)t * d + col);
+      float f[V::N];
+      v.to_float(f);
+#pragma unroll
+      for (int j = 0; j < V::N; ++j) acc[j] = fmaf(g, f[j], acc[j]);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < V::N; ++j) part[w][lane * V::N + j] = acc[j];
+  __syncthreads();
+  for (int i = threadIdx.x; i < 32 * V::N; i += blockDim.x) {
+    float s = 0.f;
+#pragma unroll
+    for (int ww = 0; ww < 8; ++ww) s += part[ww][i];
+    const int c = blockIdx.x * 32 * V::N + i;
+    if (c < d) ws[(size_t)blockIdx.y * d + c] = s;
+  }
+}
+
+__global__ void sum_splits_kernel(const float* __restrict__ ws, float* __restrict__ out, int d) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= d) return;
+  float s = 0.f;
+  for (int i = 0; i < GWS_SPLITS; ++i) s += ws[(size_t)i * d + c];
+  out[c] = s;
+}
+
+inline int perm_blocks(const c2r_config* cfg) {
+  long long NK = (long long)cfg->N * cfg->K;
+  return (int)((NK + PERM_BLOCK_SLOTS - 1) / PERM_BLOCK_SLOTS);
+}
+
+size_t permute_ws_bytes(const c2r_config* cfg) {
+  return sizeof(int32_t) * (size_t)(perm_blocks(cfg) > 0 ? perm_blocks(cfg) : 1) * cfg->E;
+}
+size_t gate_bwd_ws_bytes(const c2r_config* cfg) { return sizeof(float) * (size_t)GWS_SPLITS * cfg->d; }
+
+template <typename T>
+int permute_impl(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const T* X, int32_t* counts,
+                 int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, T* Xp, int32_t* status, void* ws,
+                 cudaStream_t s) {
+  const long long NK = (long long)cfg->N * cfg->K;
+  const long long R = permuted_rows(cfg);
+  const int nb = perm_blocks(cfg);
+  int32_t* block_counts = (int32_t*)ws;
+  C2R_CUDA(cudaMemsetAsync(slot_of_row, 0xFF, sizeof(int32_t) * R, s));
+  if (nb > 0) {
+    perm_hist_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, status);
+    C2R_LAUNCH_CHECK();
+  }
+  perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, cfg->E, expert_rank, cfg->row_align, counts, offsets);
+  C2R_LAUNCH_CHECK();
+  if (nb > 0) {
+    perm_rank_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, offsets, row_of_slot, slot_of_row);
+    C2R_LAUNCH_CHECK();
+  }
+  if (X != nullptr) {
+    if (cfg->N > 0) {
+      permute_rows_kernel<T><<<(cfg->N + 7) / 8, 256, 0, s>>>(X, row_of_slot, Xp, cfg->N, cfg->d, cfg->K);
+      C2R_LAUNCH_CHECK();
+    }
+    if (R > NK) {
+      int blocks = (int)((R + 7) / 8);
+      if (blocks > 1184) blocks = 1184;
+      zero_pad_rows_kernel<T><<<blocks, 256, 0, s>>>(slot_of_row, Xp, R, cfg->d);
+      C2R_LAUNCH_CHECK();
+    }
+  }
+  return C2R_OK;
+}
+
+}  // namespace c2r
+
+using namespace c2r;
+
+extern "C" int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
+                           int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp,
+                           int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(idx && counts && offsets && row_of_slot && slot_of_row, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!X || Xp, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(ws && ws_bytes >= permute_ws_bytes(cfg), C2R_ERR_WORKSPACE);
+  if (cfg->dtype == C2R_BF16)
+    return permute_impl<__nv_bfloat16>(cfg, idx, expert_rank, (const __nv_bfloat16*)X, counts, offsets, row_of_slot,
+                                       slot_of_row, (__nv_bfloat16*)Xp, status, ws, as_stream(stream));
+  return permute_impl<float>(cfg, idx, expert_rank, (const float*)X, counts, offsets, row_of_slot, slot_of_row,
+                             (float*)Xp, status, ws, as_stream(stream));
+}
+
+template <typename T>
+static int gather_sum_launch(const c2r_config* cfg, const void* src, const int32_t* rows, const float* coef,
+                             const void* extra, const float* z, const int32_t* idx, const float* dl, const void* Wg,
+                             const float* dz, const void* wsg, void* out, int accumulate, cudaStream_t s) {
+  if (cfg->N == 0) return C2R_OK;
+  gather_sum_kernel<T><<<(cfg->N + 7) / 8, 256, 0, s>>>((const float*)src, rows, coef, (const float*)extra, z, idx, dl,
+                                                        (const T*)Wg, dz, (const T*)wsg, (T*)out, accumulate, cfg->N,
+                                                        cfg->d, cfg->K);
+  C2R_LAUNCH_CHECK();
+  return C2R_OK;
+}
+
+extern "C" int c2r_combine(const c2r_config* cfg, const void* Yp, const float* w, const int32_t* row_of_slot,
+                           const void* Ys, const float* z, void* Y, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(Yp && w && row_of_slot && Y, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!Ys || z, C2R_ERR_INVALID_ARG);
+  if (cfg->dtype == C2R_BF16)
+    return gather_sum_launch<__nv_bfloat16>(cfg, Yp, row_of_slot, w, Ys, z, nullptr, nullptr, nullptr, nullptr,
+                                            nullptr, Y, 0, as_stream(stream));
+  return gather_sum_launch<float>(cfg, Yp, row_of_slot, w, Ys, z, nullptr, nullptr, nullptr, nullptr, nullptr, Y, 0,
+                                  as_stream(stream));
+}
+
+extern "C" int c2r_unpermute_grad(const c2r_config* cfg, const void* dXp, const int32_t* row_of_slot, const void* dXs,
+                                  const int32_t* idx, const float* dl, const void* Wg, const float* dz,
+                                  const void* wsg, void* dX, int accumulate, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(dXp && row_of_slot && dX, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!dl || (idx && Wg), C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE((dz == nullptr) == (wsg == nullptr), C2R_ERR_INVALID_ARG);
+  if (cfg->dtype == C2R_BF16)
+    return gather_sum_launch<__nv_bfloat16>(cfg, dXp, row_of_slot, nullptr, dXs, nullptr, idx, dl, Wg, dz, wsg, dX,
+                                            accumulate, as_stream(stream));
+  return gather_sum_launch<float>(cfg, dXp, row_of_slot, nullptr, dXs, nullptr, idx, dl, Wg, dz, wsg, dX, accumulate,
+                                  as_stream(stream));
+}
+
+template <typename T>
+static int combine_bwd_launch(const c2r_config* cfg, const void* dY, const void* Yp, const float* w,
+                              const int32_t* rows, const int32_t* slot_of_row, const void* Ys, const float* z,
+                              void* dYp, float* dw, void* dYs, float* dz, cudaStream_t s) {
+  const long long R = permuted_rows(cfg);
+  if (cfg->N > 0) {
+    combine_bwd_kernel<T><<<(cfg->N + 7) / 8, 256, 0, s>>>((const T*)dY, (const float*)Yp, w, rows, (const float*)Ys, z,
+                                                           (T*)dYp, dw, (T*)dYs, dz, cfg->N, cfg->d, cfg->K);
+    C2R_LAUNCH_CHECK();
+  }
+  if (R > (long long)cfg->N * cfg->K) {
+    int blocks = (int)((R + 7) / 8);
+    if (blocks > 1184) blocks = 1184;
+    zero_pad_rows_kernel<T><<<blocks, 256, 0, s>>>(slot_of_row, (T*)dYp, R, cfg->d);
+    C2R_LAUNCH_CHECK();
+  }
+  return C2R_OK;
+}
+
+extern "C" int c2r_combine_bwd(const c2r_config* cfg, const void* dY, const void* Yp, const float* w,
+                               const int32_t* row_of_slot, const int32_t* slot_of_row, const void* Ys, const float* z,
+                               void* dYp, float* dw, void* dYs, float* dz, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(dY && Yp && w && row_of_slot && slot_of_row && dYp && dw, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!Ys || (z && dYs && dz), C2R_ERR_INVALID_ARG);
+  if (cfg->dtype == C2R_BF16)
+    return combine_bwd_launch<__nv_bfloat16>(cfg, dY, Yp, w, row_of_slot, slot_of_row, Ys, z, dYp, dw, dYs, dz,
+                                             as_stream(stream));
+  return combine_bwd_launch<float>(cfg, dY, Yp, w, row_of_slot, slot_of_row, Ys, z, dYp, dw, dYs, dz,
+                                   as_stream(stream));
+}
+
+template <typename T>
+static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
+                           const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
+                           float* dWg, float* dwsg, void* ws, cudaStream_t s) {
+  using V = Vec16<T>;
+  const int colblocks = (cfg->d + 32 * V::N - 1) / (32 * V::N);
+  gate_wgrad_kernel<T><<<dim3(colblocks, cfg->E), 256, 0, s>>>((const T*)Xp, counts, offsets, slot_of_row, dl, dWg,
+                                                               cfg->d);
+  C2R_LAUNCH_CHECK();
+  if (dz) {
+    shared_gate_wgrad_kernel<T><<<dim3(colblocks, GWS_SPLITS), 256, 0, s>>>((const T*)X, dz, (float*)ws, cfg->N, cfg->d);
+    C2R_LAUNCH_CHECK();
+    sum_splits_kernel<<<(cfg->d + 255) / 256, 256, 0, s>>>((const float*)ws, dwsg, cfg->d);
+    C2R_LAUNCH_CHECK();
+  }
+  return C2R_OK;
+}
+
+extern "C" int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
+                            const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
+                            float* dWg, float* dwsg, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(Xp && counts && offsets && slot_of_row && dl && dWg, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!dz || (X && dwsg), C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!dz || (ws && ws_bytes >= gate_bwd_ws_bytes(cfg)), C2R_ERR_WORKSPACE);
+  if (cfg->dtype == C2R_BF16)
+    return gate_bwd_launch<__nv_bfloat16>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws,
+                                          as_stream(stream));
+  return gate_bwd_launch<float>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws, as_stream(stream));
+}

@@ -1,0 +1,207 @@
+"""GPU parity: floating-point steps and the whole layer against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import c2r_oracle as O
+from paper_2504_01337_b200 import inputs as G
+from tests.util import assert_close_abs, assert_close_elem, assert_close_rms, dev, host, live_rows, mask_of, random_sets
+
+pytestmark = pytest.mark.gpu
+
+
+def B():
+    from paper_2504_01337_b200 import binding
+    return binding
+
+
+def _layer(wl, **kw):
+    from paper_2504_01337_b200.layer import C2RLayer
+    return C2RLayer(wl.N, wl.d, wl.E, wl.I, wl.K, wl.T, wl.P, wl.I_s, wl.bf16, **kw)
+
+
+def _close(bf16, stored_bf16=True):
+    """Output bar: bf16 configurations 2e-2*RMS (see assert_close_rms), fp32 configurations max-abs 1e-4."""
+    return (lambda g, r, what: assert_close_rms(g, r, 2e-2, what, out_bf16=stored_bf16)) if bf16 else \
+           (lambda g, r, what: assert_close_abs(g, r, 1e-4, what))
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_gate_logits(bf16):
+    b = B()
+    N, d, E = 1000, 256, 60
+    X = G.normal(1, G.S_X, (N, d)); Wg = G.normal(1, G.S_WG, (E, d), 0.02); wsg = G.normal(1, G.S_WSG, (d,), 0.02)
+    if bf16:
+        X, Wg, wsg = G.round_bf16(X), G.round_bf16(Wg), G.round_bf16(wsg)
+    dt = torch.bfloat16 if bf16 else None
+    cfg = b.make_config(N, d, E, 16, 4, 8, 1, 16, b.BF16 if bf16 else b.F32, 1)
+    L = torch.zeros((N, E), device="cuda"); z = torch.zeros((N,), device="cuda")
+    b.gate_logits(cfg, dev(X, dt), dev(Wg, dt), dev(wsg, dt), L, z)
+    assert_close_abs(host(L), O.gate_logits(X, Wg), 1e-4, "L")
+    assert_close_abs(host(z), X.astype(np.float64) @ wsg.astype(np.float64), 1e-4, "z")
+
+
+def test_c1_layer_forward_fp32():
+    """Tiny fp32 layer: calibration batch -> Eq. 2 -> Eq. 4 sets -> placement -> C2R forward."""
+    b = B()
+    wl = G.WORKLOADS["c1"]
+    X = G.hidden(wl); Xcal = G.hidden(wl, calib=True)
+    Wg, _ = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    # profiling on the device
+    cal = b.make_config(wl.n_calib, wl.d, wl.E, wl.I, wl.K, wl.T, wl.P, 0, b.F32, 1)
+    Lc = torch.zeros((wl.n_calib, wl.E), device="cuda")
+    b.gate_logits(cal, dev(Xcal), dev(Wg), None, Lc, None)
+    idxc = torch.zeros((wl.n_calib, wl.K), dtype=torch.int32, device="cuda")
+    wc = torch.zeros((wl.n_calib, wl.K), device="cuda")
+    b.route(cal, Lc, None, idxc, wc)
+    Cm = torch.zeros((wl.E, wl.E), dtype=torch.int32, device="cuda")
+    b.collab_count(cal, idxc, wl.n_calib, Cm)
+    I_T = torch.zeros((wl.E, wl.T), dtype=torch.int32, device="cuda")
+    mask = torch.zeros((wl.E,), dtype=torch.int64, device="cuda")
+    b.collab_sets(cal, Cm, I_T, mask)
+    # oracle on the device's calibration logits (routing is compared given identical fp32 logits)
+    ridx_c, _ = O.topk_route(host(Lc), wl.K)
+    assert np.array_equal(host(idxc), ridx_c)
+    Cref = O.collab_count(ridx_c, wl.E)
+    assert np.array_equal(host(Cm), Cref)
+    sets = O.collab_sets(Cref, wl.T)
+    assert np.array_equal(host(I_T), sets)
+    part_ref, rank_ref = O.place_experts(Cref, wl.P)
+    part = torch.zeros(wl.E, dtype=torch.int32); rank = torch.zeros(wl.E, dtype=torch.int32)
+    b.place_experts(cal, Cm.cpu(), 0, part, rank)
+    assert np.array_equal(part.numpy(), part_ref) and np.array_equal(rank.numpy(), rank_ref)
+
+    lay = _layer(wl, backward=False)
+    lay.set_params(Wg, W1, W3, W2)
+    lay.set_routing(mask=host(mask).view(np.uint64), expert_rank=rank_ref, part=part_ref)
+    lay.set_input(X)
+    lay.forward()
+    torch.cuda.synchronize()
+    Lg = lay.host("L")
+    assert_close_abs(Lg, O.gate_logits(X, Wg), 1e-4, "L")
+    f = O.layer_fwd(X, Wg, W1, W3, W2, sets, wl.K, expert_rank=rank_ref, row_align=1, logits=Lg)
+    assert np.array_equal(lay.host("idx"), f["idx"])
+    assert np.array_equal(lay.host("counts"), f["counts"]) and np.array_equal(lay.host("offsets"), f["offsets"])
+    assert np.array_equal(lay.host("row_of_slot"), f["row_of_slot"])
+    assert_close_abs(lay.host("w"), f["w"], 1e-4, "w")
+    n = f["slot_of_row"].size
+    assert np.array_equal(lay.host("Xp")[:n], f["Xp"].astype(np.float32))
+    assert_close_abs(lay.host("H")[:n], f["H"], 1e-4, "H")
+    assert_close_abs(lay.host("Yp")[:n], f["Yp"], 1e-4, "Yp")
+    assert_close_abs(lay.host("Y"), f["Y"], 1e-4, "Y")
+    v = O.dispatch_volume(f["idx"], part_ref, wl.P)
+    vol = lay.host("volume")
+    assert vol[:4].tolist() == [v["naive"], v["dedup"], v["naive_x"], v["dedup_x"]]
+    assert int(lay.t["status"].item()) == 0
+
+
+SMALL = [
+    # name,           N,   d,   E,  I,   K, T, P, I_s, bf16
+    ("f32-noshared", 300, 64, 8, 48, 2, 3, 2, 0, False),
+    ("f32-shared", 257, 64, 6, 32, 3, 4, 3, 64, False),
+    ("bf16-shared", 2048, 256, 8, 400, 4, 5, 4, 528, True),
+    ("bf16-noshared", 2048, 256, 8, 384, 2, 4, 4, 0, True),
+]
+
+
+@pytest.mark.parametrize("name,N,d,E,I,K,T,P,I_s,bf16", SMALL)
+def test_small_layer_forward_backward(name, N, d, E, I, K, T, P, I_s, bf16):
+    wl = G.Workload(name, N=N, d=d, E=E, I=I, K=K, T=T, P=P, I_s=I_s, bf16=bf16, seed=11)
+    close = _close(bf16)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    # the bench recipe's weights; the gate is scaled up so that routing weights are far from uniform
+    r = (lambda a: G.round_bf16(a)) if bf16 else (lambda a: a)
+    W1, W3, W2 = G.expert_weights(wl)
+    Wg = Wg if bf16 else Wg * 8
+    sh = G.shared_weights(wl) if I_s else None
+    sets = random_sets(E, T, seed=5)
+    rank = np.random.default_rng(3).permutation(E)
+    lay = _layer(wl, backward=True)
+    lay.set_params(Wg, W1, W3, W2, wsg, sh)
+    lay.set_routing(mask=mask_of(sets, E), expert_rank=rank)
+    lay.set_input(X, dY)
+    lay.forward()
+    lay.backward()
+    torch.cuda.synchronize()
+    align = lay.cfg.row_align
+    Lg = lay.host("L")
+    f = O.layer_fwd(X, Wg, W1, W3, W2, sets, K, expert_rank=rank, row_align=align, shared=sh, wsg=wsg, logits=Lg)
+    assert np.array_equal(lay.host("idx"), f["idx"])
+    assert np.array_equal(lay.host("offsets"), f["offsets"])
+    assert np.array_equal(lay.host("row_of_slot"), f["row_of_slot"])
+    assert_close_abs(lay.host("w"), f["w"], 1e-4, "w")
+    live = live_rows(f["counts"], f["offsets"])
+    close32 = _close(bf16, stored_bf16=False)      # results the library keeps in fp32
+    mid = (lambda g, r, what: assert_close_elem(g, r, what=what)) if bf16 else close
+    mid(lay.host("H")[live], f["H"][live], "H")
+    # per-(token, expert) partials are internal: looser max bound, same RMS bound
+    part = (lambda g, r, what: assert_close_rms(g, r, 5e-2, what, out_bf16=False)) if bf16 else close
+    part(lay.host("Yp")[live], f["Yp"][live], "Yp")
+    close(lay.host("Y"), f["Y"], "Y")
+    # backward: the oracle differentiates its own forward (logits from X Wg, routing frozen)
+    f2 = O.layer_fwd(X, Wg, W1, W3, W2, sets, K, expert_rank=rank, row_align=align, shared=sh, wsg=wsg)
+    if not np.array_equal(f2["idx"], f["idx"]):
+        pytest.skip("fp32 and fp64 logits disagree on a near-tie; backward parity needs equal routing")
+    g = O.layer_bwd(X, Wg, W1, W3, W2, f2, dY, shared=sh, wsg=wsg)
+    close32(lay.host("dw"), g["dw"], "dw")
+    mid(lay.host("dYp")[live], g["dYp"][live], "dYp")
+    part(lay.host("dXp")[live], g["dXp"][live], "dXp")
+    grads = [host(t) for t in lay.unpacked_grads()]
+    close(grads[0], g["dW1"], "dW1")
+    close(grads[1], g["dW3"], "dW3")
+    close(lay.host("dW2"), g["dW2"], "dW2")
+    close32(lay.host("dWg"), g["dWg"], "dWg")
+    close(lay.host("dX"), g["dX"], "dX")
+    if I_s:
+        close32(lay.host("dz"), g["dz"], "dz")
+        close(grads[2], g["dWs1"], "dWs1")
+        close(grads[3], g["dWs3"], "dWs3")
+        close(lay.host("dWs2")[0], g["dWs2"], "dWs2")
+        close32(lay.host("dwsg"), g["dwsg"], "dwsg")
+    # padding rows of the permuted buffers are zero
+    pad = np.setdiff1d(np.arange(int(f["offsets"][E])), live)
+    if pad.size:
+        assert np.all(lay.host("Xp")[pad] == 0) and np.all(lay.host("dYp")[pad] == 0)
+
+
+def test_pack_unpack_roundtrip():
+    b = B()
+    for I in (16, 128, 144, 688):
+        E, d = 3, 64
+        cfg = b.make_config(8, d, E, I, 2, 1, 1, 0, b.BF16, 128)
+        W1 = dev(G.round_bf16(G.normal(1, G.S_W1, (E, I, d))), torch.bfloat16)
+        W3 = dev(G.round_bf16(G.normal(1, G.S_W3, (E, I, d))), torch.bfloat16)
+        Wp = torch.zeros((E, 2 * I, d), dtype=torch.bfloat16, device="cuda")
+        b.pack_weights(cfg, E, I, W1, W3, Wp)
+        ref = np.zeros((E, 2 * I, d), dtype=np.float32)
+        for j in range(0, I, 128):
+            wdt = min(128, I - j)
+            ref[:, 2 * j:2 * j + wdt] = host(W1)[:, j:j + wdt]
+            ref[:, 2 * j + wdt:2 * j + 2 * wdt] = host(W3)[:, j:j + wdt]
+        assert np.array_equal(host(Wp), ref)
+        A1 = torch.zeros_like(W1); A3 = torch.zeros_like(W3)
+        b.unpack_weights(cfg, E, I, Wp, A1, A3)
+        assert torch.equal(A1, W1) and torch.equal(A3, W3)
+
+
+def test_train_step_refreshes_sets_from_live_routing():
+    wl = G.Workload("step", N=512, d=128, E=16, I=128, K=4, T=6, P=4, I_s=128, bf16=True, seed=2)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    sh = G.shared_weights(wl)
+    sets = random_sets(wl.E, wl.T, seed=9)
+    lay = _layer(wl, backward=True, profile=True)
+    lay.set_params(Wg, W1, W3, W2, wsg, sh)
+    lay.set_routing(mask=mask_of(sets, wl.E))
+    lay.set_input(X, dY)
+    lay.train_step()
+    torch.cuda.synchronize()
+    idx = lay.host("idx").astype(np.int64)
+    Cref = O.collab_count(idx, wl.E)
+    assert np.array_equal(lay.host("C"), Cref)
+    new_sets = O.collab_sets(Cref, wl.T)
+    assert np.array_equal(lay.host("I_T"), new_sets)
+    assert np.array_equal(lay.host("mask_next").view(np.uint64), mask_of(new_sets, wl.E))

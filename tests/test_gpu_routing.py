@@ -1,0 +1,207 @@
+"""GPU parity: routing side (integer outputs bit-exact against the oracle)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import c2r_oracle as O
+from paper_2504_01337_b200 import inputs as G
+from tests.util import assert_close_abs, dev, host, mask_of, random_sets
+
+pytestmark = pytest.mark.gpu
+
+
+def B():
+    from paper_2504_01337_b200 import binding
+    return binding
+
+
+def _route_gpu(L, mask, K, T, renorm=1, want_p=False):
+    b = B()
+    N, E = L.shape
+    cfg = b.make_config(N, 8, E, 16, K, T, 1, 0, b.F32, 1, renorm)
+    Ld = dev(L.astype(np.float32))
+    idx = torch.full((N, K), -7, dtype=torch.int32, device="cuda")
+    w = torch.zeros((N, K), dtype=torch.float32, device="cuda")
+    p = torch.zeros((N, E), dtype=torch.float32, device="cuda") if want_p else None
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    md = dev(mask.view(np.int64)) if mask is not None else None
+    b.route(cfg, Ld, md, idx, w, p, status)
+    torch.cuda.synchronize()
+    return host(idx).astype(np.int64), host(w), (host(p) if want_p else None), int(status.item())
+
+
+@pytest.mark.parametrize("E,K,T", [(8, 2, 4), (16, 4, 8), (60, 4, 16), (64, 8, 20), (60, 4, 59), (33, 3, 2), (5, 1, 0), (64, 1, 5)])
+def test_route_matches_oracle(E, K, T):
+    N = 3001
+    for kind in ("normal", "ties"):
+        if kind == "normal":
+            L = G.random_logits(E * 7 + K, N, E, std=0.9)
+        else:
+            L = ((G.integers(E + K, G.S_MISC, (N, E), 5).astype(np.float32)) - 2.0) * 0.25
+        I_T = random_sets(E, T, seed=E + T)
+        mask = mask_of(I_T, E)
+        idx, w, _, st = _route_gpu(L, mask, K, T)
+        ridx, rw = O.c2r_route(L, I_T, K)
+        assert np.array_equal(idx, ridx)
+        assert_close_abs(w, rw, 1e-6, "w")
+        assert st == 0
+        idx, w, p, _ = _route_gpu(L, None, K, T, want_p=True)
+        ridx, rw = O.topk_route(L, K)
+        assert np.array_equal(idx, ridx)
+        assert_close_abs(w, rw, 1e-6, "w topk")
+        assert_close_abs(p, O.softmax_rows(L), 1e-6, "p")
+        idx, w, _, _ = _route_gpu(L, None, K, T, renorm=0)
+        assert_close_abs(w, O.route_weights(L, ridx, renorm=False), 1e-6, "w no renorm")
+
+
+def test_route_nonfinite_and_zero_sign():
+    E, K = 8, 3
+    L = G.random_logits(3, 64, E)
+    L[0, :] = -np.inf
+    L[1, 2] = np.nan
+    L[2, :] = 0.0
+    L[2, 3] = -0.0
+    L[3, 5] = np.inf
+    idx, w, _, st = _route_gpu(L, None, K, 0)
+    ridx, _ = O.topk_route(L, K)
+    assert np.array_equal(idx, ridx)
+    assert st & 1
+
+
+def test_route_set_too_small_is_flagged_not_fatal():
+    E, K = 8, 4
+    L = G.random_logits(4, 100, E)
+    mask = np.array([1 << ((i + 1) % E) for i in range(E)], dtype=np.uint64)  # one collaborator, K-1 = 3 needed
+    idx, w, _, st = _route_gpu(L, mask, K, 3)
+    assert st & 2
+    assert all(len(set(r)) == K for r in idx.tolist())
+    assert np.array_equal(idx[:, 0], np.argmax(L, axis=1))
+
+
+@pytest.mark.parametrize("E,K,N", [(8, 2, 4096), (60, 4, 16384), (64, 8, 1000), (16, 4, 1)])
+def test_collab_count_and_sets(E, K, N):
+    b = B()
+    idx, _ = O.topk_route(G.random_logits(E + N, N, E), K)
+    T = min(E - 1, max(K - 1, E // 4))
+    cfg = b.make_config(N, 8, E, 16, K, T, 1, 0, b.F32, 1)
+    idxd = dev(idx.astype(np.int32))
+    Cd = torch.full((E, E), 99, dtype=torch.int32, device="cuda")
+    b.collab_count(cfg, idxd, N, Cd, False)
+    Cref = O.collab_count(idx, E)
+    assert np.array_equal(host(Cd), Cref)
+    b.collab_count(cfg, idxd, N // 2, Cd, True)
+    assert np.array_equal(host(Cd), Cref + O.collab_count(idx[: N // 2], E))
+    b.collab_count(cfg, idxd, N, Cd, False)
+    I_T = torch.zeros((E, T), dtype=torch.int32, device="cuda")
+    mask = torch.zeros((E,), dtype=torch.int64, device="cuda")
+    b.collab_sets(cfg, Cd, I_T, mask)
+    ref_sets = O.collab_sets(Cref, T)
+    assert np.array_equal(host(I_T), ref_sets)
+    assert np.array_equal(host(mask).view(np.uint64), mask_of(ref_sets, E))
+
+
+def test_collab_sets_with_ties_and_zero_rows():
+    b = B()
+    E, T = 12, 5
+    Cm = np.zeros((E, E), dtype=np.int32)
+    Cm[0, :] = 7
+    Cm[1, [2, 5, 9]] = [3, 3, 3]
+    Cm[3, 3] = 1000
+    cfg = b.make_config(1, 8, E, 16, 2, T, 1, 0, b.F32, 1)
+    I_T = torch.zeros((E, T), dtype=torch.int32, device="cuda")
+    mask = torch.zeros((E,), dtype=torch.int64, device="cuda")
+    b.collab_sets(cfg, dev(Cm), I_T, mask)
+    assert np.array_equal(host(I_T), O.collab_sets(Cm, T))
+
+
+@pytest.mark.parametrize("E,K,N,P", [(8, 2, 512, 2), (60, 4, 16384, 4), (60, 4, 5000, 8), (16, 4, 777, 16), (6, 3, 10, 1)])
+def test_dispatch_volume(E, K, N, P):
+    b = B()
+    idx, _ = O.topk_route(G.random_logits(E * P + N, N, E), K)
+    rng = np.random.default_rng(P)
+    part = rng.integers(0, P, E)
+    cfg = b.make_config(N, 8, E, 16, K, K - 1, P, 0, b.F32, 1)
+    tot = torch.full((4,), 5, dtype=torch.int64, device="cuda")
+    sn = torch.full((P, P), 5, dtype=torch.int64, device="cuda")
+    sd = torch.full((P, P), 5, dtype=torch.int64, device="cuda")
+    b.dispatch_volume(cfg, dev(idx.astype(np.int32)), dev(part.astype(np.int32)), tot, sn, sd)
+    v = O.dispatch_volume(idx, part, P)
+    assert host(tot).tolist() == [v["naive"], v["dedup"], v["naive_x"], v["dedup_x"]]
+    assert np.array_equal(host(sn), v["send_naive"]) and np.array_equal(host(sd), v["send_dedup"])
+
+
+@pytest.mark.parametrize("E,K,N,align", [(8, 2, 512, 1), (60, 4, 16384, 128), (60, 4, 3001, 128), (16, 4, 130, 8), (64, 8, 77, 128), (5, 1, 1, 1)])
+def test_permute_index_and_rows(E, K, N, align):
+    b = B()
+    d = 64
+    idx, _ = O.topk_route(G.random_logits(E + N + align, N, E), K)
+    rank = np.random.default_rng(E).permutation(E)
+    X = G.normal(0, G.S_X, (N, d))
+    for use_rank in (False, True):
+        for bf16 in (False, True):
+            cfg = b.make_config(N, d, E, 16, K, K - 1, 1, 0, b.BF16 if bf16 else b.F32, align)
+            R = b.permuted_rows(cfg)
+            Xh = G.round_bf16(X) if bf16 else X
+            Xd = dev(Xh, torch.bfloat16 if bf16 else None)
+            counts = torch.zeros(E, dtype=torch.int32, device="cuda")
+            offsets = torch.zeros(E + 1, dtype=torch.int32, device="cuda")
+            ros = torch.zeros(N * K, dtype=torch.int32, device="cuda")
+            sor = torch.zeros(R, dtype=torch.int32, device="cuda")
+            Xp = torch.full((R, d), 3.0, dtype=Xd.dtype, device="cuda")
+            ws = torch.empty(b.workspace_bytes(cfg, b.WS_PERMUTE), dtype=torch.uint8, device="cuda")
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            b.permute(cfg, dev(idx.astype(np.int32)), dev(rank.astype(np.int32)) if use_rank else None, Xd, counts,
+                      offsets, ros, sor, Xp, status, ws)
+            rc, ro, rros, rsor = O.permute_index(idx, E, rank if use_rank else None, align)
+            assert np.array_equal(host(counts), rc) and np.array_equal(host(offsets), ro)
+            assert np.array_equal(host(ros), rros)
+            got_sor = host(sor)
+            assert np.array_equal(got_sor[: rsor.size], rsor) and np.all(got_sor[rsor.size:] == -1)
+            ref_Xp = np.zeros((R, d), dtype=np.float32)
+            ref_Xp[: rsor.size] = O.permute(Xh, rsor, K)
+            assert np.array_equal(host(Xp), ref_Xp)
+            assert int(status.item()) == 0
+
+
+def test_permute_empty_batch_and_bad_index():
+    b = B()
+    E, K, d = 8, 2, 32
+    cfg = b.make_config(0, d, E, 16, K, 1, 1, 0, b.F32, 4)
+    R = b.permuted_rows(cfg)
+    counts = torch.ones(E, dtype=torch.int32, device="cuda")
+    offsets = torch.ones(E + 1, dtype=torch.int32, device="cuda")
+    ws = torch.empty(max(1, b.workspace_bytes(cfg, b.WS_PERMUTE)), dtype=torch.uint8, device="cuda")
+    empty = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.permute(cfg, empty, None, None, counts, offsets, empty, torch.zeros(max(R, 1), dtype=torch.int32, device="cuda"),
+              None, None, ws)
+    assert host(counts).sum() == 0 and host(offsets).sum() == 0
+    # out-of-range expert ids are clamped and reported, never dereferenced
+    N = 40
+    cfg = b.make_config(N, d, E, 16, K, 1, 1, 0, b.F32, 1)
+    idx = np.random.default_rng(0).integers(0, E, (N, K)).astype(np.int32)
+    idx[3, 1] = 99
+    idx[7, 0] = -5
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ros = torch.zeros(N * K, dtype=torch.int32, device="cuda")
+    sor = torch.zeros(b.permuted_rows(cfg), dtype=torch.int32, device="cuda")
+    b.permute(cfg, dev(idx), None, None, counts, offsets, ros, sor, None, status, ws)
+    assert int(status.item()) & 4
+    fixed = np.clip(idx, 0, E - 1)
+    assert np.array_equal(host(ros), O.permute_index(fixed, E)[2])
+
+
+def test_argument_errors_are_codes_not_faults():
+    b = B()
+    cfg = b.make_config(16, 64, 8, 16, 2, 4, 2, 0, b.F32, 1)
+    with pytest.raises(b.C2RError) as e:
+        b.route(cfg, None, None, None, None)
+    assert e.value.code == -1
+    bad = b.make_config(16, 64, 80, 16, 2, 4, 2, 0, b.F32, 1)
+    L = torch.zeros((16, 80), device="cuda")
+    with pytest.raises(b.C2RError) as e:
+        b.route(bad, L, None, torch.zeros((16, 2), dtype=torch.int32, device="cuda"), torch.zeros((16, 2), device="cuda"))
+    assert e.value.code == -2
+    idx = torch.zeros((16, 2), dtype=torch.int32, device="cuda")
+    with pytest.raises(b.C2RError) as e:
+        b.permute(cfg, idx, None, None, idx, idx, idx, idx, None, None, None)
+    assert e.value.code == -3

@@ -1,0 +1,79 @@
+"""Helpers shared by the GPU parity tests."""
+import numpy as np
+import torch
+
+from oracle import c2r_oracle as O
+from paper_2504_01337_b200 import inputs as G
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.cuda()
+
+
+def host(t):
+    return (t.float() if t.dtype == torch.bfloat16 else t).cpu().numpy()
+
+
+def assert_close_rms(got, ref, frac=2e-2, what="", out_bf16=True, rms_frac=5e-3):
+    """bf16 bar.  Every element: |err| <= frac * RMS(ref) + 2^-8 |ref|, where the second term is the
+    representation error of a bf16-stored result (half an ulp, which no implementation can avoid;
+    dropped with out_bf16=False for results stored in fp32).  And over the tensor:
+    RMS(err) <= rms_frac * RMS(ref)."""
+    got = np.asarray(got, np.float64); ref = np.asarray(ref, np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    assert np.isfinite(got).all(), what
+    if ref.size == 0:
+        return
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    err = np.abs(got - ref)
+    tol = frac * rms + (2.0 ** -8 * np.abs(ref) if out_bf16 else 0.0)
+    worst = float(np.max(err - tol))
+    assert worst <= 0.0, f"{what}: max|err|={err.max():.3e} ({err.max() / rms:.4f} RMS), over tolerance by {worst:.3e}"
+    erms = float(np.sqrt(np.mean(err ** 2)))
+    assert erms <= rms_frac * rms, f"{what}: RMS(err)={erms:.3e} > {rms_frac}*RMS(ref)={rms_frac * rms:.3e}"
+
+
+def assert_close_abs(got, ref, tol=1e-4, what=""):
+    """fp32 bar: max |err| <= tol."""
+    got = np.asarray(got, np.float64); ref = np.asarray(ref, np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    err = float(np.max(np.abs(got - ref))) if ref.size else 0.0
+    assert np.isfinite(got).all(), what
+    assert err <= tol, f"{what}: max|err|={err:.3e} > {tol}"
+
+
+def assert_close_elem(got, ref, rel=2.0 ** -7, abs_frac=2e-3, what=""):
+    """Stored bf16 intermediates (not outputs): each element within a few bf16 ulps of the reference."""
+    got = np.asarray(got, np.float64); ref = np.asarray(ref, np.float64)
+    assert got.shape == ref.shape, (what, got.shape, ref.shape)
+    rms = float(np.sqrt(np.mean(ref ** 2))) if ref.size else 0.0
+    bad = np.abs(got - ref) > rel * np.abs(ref) + abs_frac * rms + 1e-30
+    assert np.isfinite(got).all() and not bad.any(), f"{what}: {int(bad.sum())} elements off"
+
+
+def random_sets(E, T, seed):
+    rng = np.random.default_rng(seed)
+    return np.stack([rng.permutation([j for j in range(E) if j != i])[:T] for i in range(E)]).astype(np.int64)
+
+
+def mask_of(I_T, E):
+    return O.member_to_mask(O.sets_to_member(I_T, E))
+
+
+def small_layer_inputs(wl, scale_w=None):
+    """numpy inputs of a workload (bf16-rounded when wl.bf16)."""
+    X = G.hidden(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    sh = G.shared_weights(wl)
+    return X, Wg, wsg, W1, W3, W2, sh
+
+
+def live_rows(counts, offsets):
+    rows = []
+    for e in range(len(counts)):
+        rows.extend(range(int(offsets[e]), int(offsets[e]) + int(counts[e])))
+    return np.array(rows, dtype=np.int64)
