@@ -137,10 +137,13 @@ int c2r_unpack_weights(const c2r_config* cfg, int n_experts, int I, const void* 
  * W2 [n_experts, d, I] T.  out: AB [R, 2I] T (A and B in the packed column layout, kept for the
  * backward pass), H [R,I] T, Yp [R,d] float.
  * R = rows of the buffers.  Padding rows of Xp must be zero.  n_experts = 1 with counts = {R},
- * offsets = {0,R} evaluates the dense shared expert. */
+ * offsets = {0,R} evaluates the dense shared expert.
+ * bf16 runs on the tensor cores (tcgen05) when d % 16 == 0 and, for n_experts > 1, row_align is a
+ * multiple of 128; other shapes and fp32 use a CUDA-core kernel.  status (one int32, may be NULL)
+ * receives C2R_STATUS_WAIT_TIMEOUT if a bounded wait inside the kernel gave up (results invalid). */
 int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                            const int32_t* counts, const int32_t* offsets, const void* W13p,
-                           const void* W2, void* AB, void* H, void* Yp, void* stream);
+                           const void* W2, void* AB, void* H, void* Yp, int32_t* status, void* stream);
 
 /* Backward of the above:  dH = dYp W2; dA = dH * B * silu'(A); dB = dH * silu(A);
  * dXp = dA W1 + dB W3; dW2_e = dYp^T H; dW1_e = dA^T Xp; dW3_e = dB^T Xp.
@@ -150,7 +153,7 @@ int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int I, int64_t 
 int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                            const int32_t* counts, const int32_t* offsets, const void* W13p,
                            const void* W2, const void* AB, const void* H, const void* dYp, void* dAB,
-                           void* dXp, void* dW13p, void* dW2, int accumulate, void* stream);
+                           void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status, void* stream);
 
 /* Sec. 3.1 (weighted sum of the selected experts' outputs):
  * Y[t,:] = sum_k w[t,k] * Yp[row_of_slot[t*K+k],:]  (k ascending, fp32)

@@ -74,8 +74,8 @@ _SIGS = {
     "c2r_permute": [_CFG] + [_P] * 10 + [C.c_size_t, _P],
     "c2r_pack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
     "c2r_unpack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
-    "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 9,
-    "c2r_grouped_swiglu_bwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 12 + [C.c_int, _P],
+    "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 10,
+    "c2r_grouped_swiglu_bwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 12 + [C.c_int, _P, _P],
     "c2r_combine": [_CFG] + [_P] * 7,
     "c2r_combine_bwd": [_CFG] + [_P] * 12,
     "c2r_route_bwd": [_CFG] + [_P] * 4,
@@ -168,16 +168,16 @@ def unpack_weights(cfg, n_experts, I, W13p, W1, W3):
     _call("c2r_unpack_weights", C.byref(cfg), n_experts, I, _ptr(W13p), _ptr(W1), _ptr(W3), _stream())
 
 
-def grouped_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp):
+def grouped_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, status=None):
     _call("c2r_grouped_swiglu_fwd", C.byref(cfg), n_experts, I, int(R), _ptr(Xp), _ptr(counts), _ptr(offsets),
-          _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(Yp), _stream())
+          _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(Yp), _ptr(status), _stream())
 
 
 def grouped_swiglu_bwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p, dW2,
-                       accumulate=False):
+                       accumulate=False, status=None):
     _call("c2r_grouped_swiglu_bwd", C.byref(cfg), n_experts, I, int(R), _ptr(Xp), _ptr(counts), _ptr(offsets),
           _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2),
-          int(accumulate), _stream())
+          int(accumulate), _ptr(status), _stream())
 
 
 def combine(cfg, Yp, w, row_of_slot, Ys, z, Y):

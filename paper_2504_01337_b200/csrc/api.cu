@@ -72,7 +72,7 @@ static int check_gemm_args(const c2r_config* cfg, int nE, int I, int64_t R) {
 
 extern "C" int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                                       const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
-                                      void* AB, void* H, void* Yp, void* stream) {
+                                      void* AB, void* H, void* Yp, int32_t* status, void* stream) {
   int rc = check_gemm_args(cfg, n_experts, I, R);
   if (rc) return rc;
   C2R_REQUIRE(Xp && counts && offsets && W13p && W2 && H && Yp, C2R_ERR_INVALID_ARG);
@@ -83,13 +83,15 @@ extern "C" int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int 
     return simt_swiglu_fwd<float>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, s);
   }
   C2R_REQUIRE(AB, C2R_ERR_INVALID_ARG);
+  if (tc_supported(cfg, n_experts, I, R))
+    return tc_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, status, s);
   return simt_swiglu_fwd<__nv_bfloat16>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, s);
 }
 
 extern "C" int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                                       const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
                                       const void* AB, const void* H, const void* dYp, void* dAB, void* dXp,
-                                      void* dW13p, void* dW2, int accumulate, void* stream) {
+                                      void* dW13p, void* dW2, int accumulate, int32_t* status, void* stream) {
   int rc = check_gemm_args(cfg, n_experts, I, R);
   if (rc) return rc;
   C2R_REQUIRE(Xp && counts && offsets && W13p && W2 && AB && H && dYp && dAB && dXp && dW13p && dW2,
@@ -98,6 +100,9 @@ extern "C" int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int 
   if (cfg->dtype == C2R_F32)
     return simt_swiglu_bwd<float>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p,
                                   dW2, accumulate, s);
+  if (tc_supported(cfg, n_experts, I, R))
+    return tc_swiglu_bwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p, dW2,
+                         accumulate, status, s);
   return simt_swiglu_bwd<__nv_bfloat16>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp,
                                         dW13p, dW2, accumulate, s);
 }
@@ -126,10 +131,10 @@ extern "C" int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
   C2R_TRY(c2r_permute(cfg, b->idx, b->expert_rank, b->X, b->counts, b->offsets, b->row_of_slot, b->slot_of_row, b->Xp,
                       b->status, b->ws, b->ws_bytes, stream));
   C2R_TRY(c2r_grouped_swiglu_fwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
-                                 b->Yp, stream));
+                                 b->Yp, b->status, stream));
   if (shared)
     C2R_TRY(c2r_grouped_swiglu_fwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
-                                   b->Hs, b->Ys, stream));
+                                   b->Hs, b->Ys, b->status, stream));
   C2R_TRY(c2r_combine(cfg, b->Yp, b->w, b->row_of_slot, shared ? b->Ys : nullptr, shared ? b->z : nullptr, b->Y,
                       stream));
   if (b->part && b->volume) {
@@ -155,10 +160,10 @@ extern "C" int c2r_layer_bwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
                           shared ? b->z : nullptr, b->dYp, b->dw, shared ? b->dYs : nullptr,
                           shared ? b->dz : nullptr, stream));
   C2R_TRY(c2r_grouped_swiglu_bwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
-                                 b->dYp, b->dAB, b->dXp, b->dW13p, b->dW2, accumulate, stream));
+                                 b->dYp, b->dAB, b->dXp, b->dW13p, b->dW2, accumulate, b->status, stream));
   if (shared)
     C2R_TRY(c2r_grouped_swiglu_bwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
-                                   b->Hs, b->dYs, b->dABs, b->dXs, b->dWs13p, b->dWs2, accumulate, stream));
+                                   b->Hs, b->dYs, b->dABs, b->dXs, b->dWs13p, b->dWs2, accumulate, b->status, stream));
   C2R_TRY(c2r_route_bwd(cfg, b->w, b->dw, b->dl, stream));
   C2R_TRY(c2r_gate_bwd(cfg, b->X, b->Xp, b->counts, b->offsets, b->slot_of_row, b->dl, shared ? b->dz : nullptr,
                        b->dWg, shared ? b->dwsg : nullptr, ws_gate, align256(gate_bwd_ws_bytes(cfg)), stream));

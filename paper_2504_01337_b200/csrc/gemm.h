@@ -37,6 +37,18 @@ int simt_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void*
                     const int32_t* offsets, const void* W13p, const void* W2, const void* AB, const void* H,
                     const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, cudaStream_t s);
 
+// Tensor-core (tcgen05) path, bf16 only.
+enum { TC_ROWS = 0, TC_WGRAD = 1 };
+enum { TC_EPI_SWIGLU_FWD = 0, TC_EPI_F32 = 1, TC_EPI_SWIGLU_BWD = 2, TC_EPI_WGRAD_BF16 = 3 };
+bool tc_supported(const c2r_config* cfg, int nE, int I, int64_t R);
+int tc_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
+                  const int32_t* offsets, const void* W13p, const void* W2, void* AB, void* H, void* Yp,
+                  int32_t* status, cudaStream_t s);
+int tc_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
+                  const int32_t* offsets, const void* W13p, const void* W2, const void* AB, const void* H,
+                  const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status,
+                  cudaStream_t s);
+
 size_t permute_ws_bytes(const c2r_config* cfg);
 size_t gate_bwd_ws_bytes(const c2r_config* cfg);
 
