@@ -34,7 +34,8 @@ typedef enum c2r_error {
   C2R_ERR_INVALID_ARG = -1,       /* NULL where a buffer is required, or a value out of range */
   C2R_ERR_UNSUPPORTED_SHAPE = -2, /* a documented shape limit is violated */
   C2R_ERR_WORKSPACE = -3,         /* workspace missing or smaller than c2r_workspace_bytes() */
-  C2R_ERR_CUDA = -4               /* a CUDA runtime / driver call failed */
+  C2R_ERR_CUDA = -4,              /* a CUDA runtime / driver call failed */
+  C2R_ERR_STATIC_SCRATCH = -5     /* c2r_permute_static: the batch needs more than the built-in scratch */
 } c2r_error;
 
 enum { C2R_F32 = 0, C2R_BF16 = 1 };
@@ -119,6 +120,31 @@ int c2r_place_experts(const c2r_config* cfg, const int32_t* C_host, int mode, in
 int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
                 int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp,
                 int32_t* status, void* ws, size_t ws_bytes, void* stream);
+
+/* c2r_permute without a workspace argument (an addition of this library; the paper has no
+ * counterpart).  Same inputs, same outputs and the same bit-exact results as c2r_permute; the
+ * only difference is where the per-block expert counts live: in a fixed array of
+ * C2R_PERMUTE_STATIC_SCRATCH_BYTES that is part of the library's device image, so the call (like
+ * every call here) performs no cudaMalloc / cudaFree and the caller needs no scratch buffer either.
+ *
+ * Who needs it: callers that have no way to obtain device scratch at the point of the call --
+ * a serving process whose device memory has been handed in full to its own pool, a plug-in
+ * running under a host that forbids allocation on its hot path, or code in a latency-critical
+ * section where cudaMalloc's device-wide synchronisation is not acceptable.
+ *
+ * Limit: ceil(N*K / 512) * E * 4 bytes must fit the array, i.e. about N*K <= 2.0 M slots at
+ * E = 64; a larger batch is refused with C2R_ERR_STATIC_SCRATCH before anything is enqueued.
+ * Cost: every GPU that loads the library carries the array (1 MiB) until the process exits.
+ * Set-up: the first call on each device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array.  It keeps the previous call's contents,
+ * which is harmless (each call writes every entry before reading it), but two calls whose
+ * kernels can overlap on the GPU -- different streams, or different host threads on
+ * unordered streams -- race on it and must be ordered by the caller. */
+#define C2R_PERMUTE_STATIC_SCRATCH_BYTES (1u << 20)
+int c2r_permute_static(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
+                       int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp,
+                       int32_t* status, void* stream);
 
 /* Weight layout used by the fused SwiGLU kernels (no counterpart in the paper).
  * W1 (gate projection) and W3 (up projection), both [n_experts, I, d] T, are interleaved in

@@ -21,7 +21,8 @@ lib = C.CDLL(LIB_PATH)
 
 F32, BF16 = 0, 1
 WS_PERMUTE, WS_GATE_BWD, WS_LAYER = 0, 1, 2
-ERRORS = {-1: "C2R_ERR_INVALID_ARG", -2: "C2R_ERR_UNSUPPORTED_SHAPE", -3: "C2R_ERR_WORKSPACE", -4: "C2R_ERR_CUDA"}
+ERRORS = {-1: "C2R_ERR_INVALID_ARG", -2: "C2R_ERR_UNSUPPORTED_SHAPE", -3: "C2R_ERR_WORKSPACE", -4: "C2R_ERR_CUDA",
+          -5: "C2R_ERR_STATIC_SCRATCH"}
 
 
 class C2RError(RuntimeError):
@@ -55,7 +56,7 @@ EXPORTS = [
     "c2r_collab_count", "c2r_collab_sets", "c2r_place_experts", "c2r_permute", "c2r_pack_weights",
     "c2r_unpack_weights", "c2r_grouped_swiglu_fwd", "c2r_grouped_swiglu_bwd", "c2r_combine", "c2r_combine_bwd",
     "c2r_route_bwd", "c2r_gate_bwd", "c2r_unpermute_grad", "c2r_dispatch_volume", "c2r_layer_fwd",
-    "c2r_layer_bwd", "c2r_train_step",
+    "c2r_layer_bwd", "c2r_train_step", "c2r_permute_static",
 ]
 
 _P = C.c_void_p
@@ -72,6 +73,7 @@ _SIGS = {
     "c2r_collab_sets": [_CFG] + [_P] * 4,
     "c2r_place_experts": [_CFG, _P, C.c_int, _P, _P],
     "c2r_permute": [_CFG] + [_P] * 10 + [C.c_size_t, _P],
+    "c2r_permute_static": [_CFG] + [_P] * 10,
     "c2r_pack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
     "c2r_unpack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
     "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 10,
@@ -158,6 +160,12 @@ def permute(cfg, idx, expert_rank, X, counts, offsets, row_of_slot, slot_of_row,
     _call("c2r_permute", C.byref(cfg), _ptr(idx), _ptr(expert_rank), _ptr(X), _ptr(counts), _ptr(offsets),
           _ptr(row_of_slot), _ptr(slot_of_row), _ptr(Xp), _ptr(status), _ptr(ws),
           0 if ws is None else ws.numel() * ws.element_size(), _stream())
+
+
+def permute_static(cfg, idx, expert_rank, X, counts, offsets, row_of_slot, slot_of_row, Xp, status):
+    """c2r_permute with the scratch inside the library (no workspace, no allocation anywhere)."""
+    _call("c2r_permute_static", C.byref(cfg), _ptr(idx), _ptr(expert_rank), _ptr(X), _ptr(counts), _ptr(offsets),
+          _ptr(row_of_slot), _ptr(slot_of_row), _ptr(Xp), _ptr(status), _stream())
 
 
 def pack_weights(cfg, n_experts, I, W1, W3, W13p):

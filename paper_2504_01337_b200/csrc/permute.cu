@@ -608,3 +608,56 @@ extern "C" int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp
                                           as_stream(stream));
   return gate_bwd_launch<float>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws, as_stream(stream));
 }
+
+// ---------------------------------------------------------------------------------------------
+// c2r_permute_static: the same dispatch with its scratch in this library's own device image.
+// ---------------------------------------------------------------------------------------------
+namespace c2r {
+
+constexpr size_t PERM_STATIC_INTS = C2R_PERMUTE_STATIC_SCRATCH_BYTES / sizeof(int32_t);
+
+// Per-block expert counts of c2r_permute_static.  One copy lives on every GPU that loads the
+// library, from load until the process exits.  Nothing in it has to start at zero: each call
+// writes every entry it later reads (the histogram kernel stores all E counts of every block it
+// launches), so the leftovers of the previous call are never observed.
+static __device__ __align__(256) int32_t g_perm_static_scratch[PERM_STATIC_INTS];
+
+// Device address of the array above on the current device.  In host code the array's name only
+// stands for the symbol; the address a kernel can use has to be asked for, per device.
+static int perm_static_scratch(int32_t** out) {
+  constexpr int MAX_DEV = 64;
+  static int32_t* cache[MAX_DEV] = {};
+  int dev = 0;
+  C2R_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEV) return C2R_ERR_UNSUPPORTED_SHAPE;
+  int32_t* p = __atomic_load_n(&cache[dev], __ATOMIC_ACQUIRE);
+  if (p == nullptr) {
+    void* addr = nullptr;
+    C2R_CUDA(cudaGetSymbolAddress(&addr, g_perm_static_scratch));
+    p = static_cast<int32_t*>(addr);
+    __atomic_store_n(&cache[dev], p, __ATOMIC_RELEASE);  // racing first calls store the same value
+  }
+  *out = p;
+  return C2R_OK;
+}
+
+}  // namespace c2r
+
+extern "C" int c2r_permute_static(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
+                                  int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row,
+                                  void* Xp, int32_t* status, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(idx && counts && offsets && row_of_slot && slot_of_row, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!X || Xp, C2R_ERR_INVALID_ARG);
+  // the scratch holds one int32 per (block of 512 slots, expert)
+  if (permute_ws_bytes(cfg) > C2R_PERMUTE_STATIC_SCRATCH_BYTES) return C2R_ERR_STATIC_SCRATCH;
+  int32_t* scratch = nullptr;
+  rc = perm_static_scratch(&scratch);
+  if (rc) return rc;
+  if (cfg->dtype == C2R_BF16)
+    return permute_impl<__nv_bfloat16>(cfg, idx, expert_rank, (const __nv_bfloat16*)X, counts, offsets, row_of_slot,
+                                       slot_of_row, (__nv_bfloat16*)Xp, status, scratch, as_stream(stream));
+  return permute_impl<float>(cfg, idx, expert_rank, (const float*)X, counts, offsets, row_of_slot, slot_of_row,
+                             (float*)Xp, status, scratch, as_stream(stream));
+}
