@@ -46,16 +46,23 @@ def measured_peaks():
 
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    Q = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
 
     def __init__(self, index):
         self.index, self.proc, self.lines = index, None, []
+        self.t0 = self.t1 = None
+
+    def mark_begin(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -74,21 +81,29 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        import datetime
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             p = [x.strip() for x in ln.split(",")]
-            if len(p) < 6:
+            if len(p) < 8:
                 continue
             try:
-                sm.append(float(p[0])); mx.append(float(p[1]))
+                ts = datetime.datetime.strptime(p[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if self.t0 is not None and not (self.t0 - 0.05 <= ts <= self.t1 + 0.05):
+                    continue  # keep only samples taken while the timed region ran
+                sm.append(float(p[1])); mx.append(float(p[2]))
             except ValueError:
                 continue
-            for n, v in zip(names, p[2:6]):
+            try:
+                pw.append(float(p[7]))
+            except ValueError:
+                pass
+            for n, v in zip(names, p[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons)}
 
 
 def build_layer(wl, device, profile=True):
@@ -248,9 +263,9 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c5"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c3s", "c5"])
     ap.add_argument("--impl", default="c2r", choices=["c2r", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=256)
     ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)
@@ -301,12 +316,13 @@ def main():
     lib_launches = getattr(B.lib, "c2r_launch_count", None)
 
     # ---- device-resident timing ----------------------------------------------------------------
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(max(args.warmup, 3)):
         lay.train_step()
     torch.cuda.synchronize()
     barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
+    sampler.mark_begin()
     launches0 = int(lib_launches()) if lib_launches else 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
@@ -315,6 +331,7 @@ def main():
         lay.train_step()
     e1.record()
     torch.cuda.synchronize()
+    sampler.mark_end()
     barrier()
     launches = (int(lib_launches()) - launches0) if lib_launches else None
     clocks = sampler.stop()

@@ -75,6 +75,9 @@ int64_t c2r_permuted_rows(const c2r_config* cfg);
 /* cudaError_t of the last failed CUDA call made by this library on the calling thread. */
 int c2r_last_cuda_error(void);
 
+/* Number of kernels this library has launched in this process (all threads, all streams). */
+uint64_t c2r_launch_count(void);
+
 /* Sec. 3.1, Eq. 1 (argument of Top-K): L[t,e] = <X[t,:], Wg[e,:]>.
  * X [N,d] T; Wg [E,d] T; wsg [d] T or NULL (gate vector of the shared expert);
  * out: L [N,E] float; z [N] float = <X[t,:], wsg> (required iff wsg != NULL). */

@@ -52,7 +52,7 @@ class LayerBuffers(C.Structure):
 
 
 EXPORTS = [
-    "c2r_workspace_bytes", "c2r_permuted_rows", "c2r_last_cuda_error", "c2r_gate_logits", "c2r_route",
+    "c2r_workspace_bytes", "c2r_permuted_rows", "c2r_last_cuda_error", "c2r_launch_count", "c2r_gate_logits", "c2r_route",
     "c2r_collab_count", "c2r_collab_sets", "c2r_place_experts", "c2r_permute", "c2r_pack_weights",
     "c2r_unpack_weights", "c2r_grouped_swiglu_fwd", "c2r_grouped_swiglu_bwd", "c2r_combine", "c2r_combine_bwd",
     "c2r_route_bwd", "c2r_gate_bwd", "c2r_unpermute_grad", "c2r_dispatch_volume", "c2r_layer_fwd",
@@ -66,6 +66,7 @@ lib.c2r_workspace_bytes.argtypes = [_CFG, C.c_int]
 lib.c2r_permuted_rows.restype = C.c_int64
 lib.c2r_permuted_rows.argtypes = [_CFG]
 lib.c2r_last_cuda_error.restype = C.c_int
+lib.c2r_launch_count.restype = C.c_uint64
 _SIGS = {
     "c2r_gate_logits": [_CFG] + [_P] * 6,
     "c2r_route": [_CFG] + [_P] * 7,

@@ -10,6 +10,7 @@
 namespace c2r {
 
 extern thread_local int g_last_cuda_error;
+extern unsigned long long g_launch_count;  // kernels launched by this library in this process
 
 inline int cuda_fail(cudaError_t e) {
   g_last_cuda_error = (int)e;
@@ -22,7 +23,11 @@ inline int cuda_fail(cudaError_t e) {
     if (_e != cudaSuccess) return ::c2r::cuda_fail(_e); \
   } while (0)
 
-#define C2R_LAUNCH_CHECK() C2R_CUDA(cudaGetLastError())
+#define C2R_LAUNCH_CHECK()                                        \
+  do {                                                            \
+    __atomic_fetch_add(&::c2r::g_launch_count, 1ull, __ATOMIC_RELAXED); \
+    C2R_CUDA(cudaGetLastError());                                 \
+  } while (0)
 
 #define C2R_REQUIRE(cond, code) \
   do {                          \

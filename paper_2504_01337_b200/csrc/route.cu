@@ -6,6 +6,7 @@
 namespace c2r {
 
 thread_local int g_last_cuda_error = 0;
+unsigned long long g_launch_count = 0;
 
 // ---------------------------------------------------------------------------------------------
 // Gate logits (Eq. 1): L = X Wg^T, z = X wsg.  CUDA-core kernel: a block owns TM tokens and all
@@ -260,6 +261,8 @@ __global__ void __launch_bounds__(256) dispatch_volume_kernel(const int32_t* __r
 using namespace c2r;
 
 extern "C" int c2r_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" uint64_t c2r_launch_count(void) { return __atomic_load_n(&g_launch_count, __ATOMIC_RELAXED); }
 
 extern "C" int c2r_gate_logits(const c2r_config* cfg, const void* X, const void* Wg, const void* wsg, float* L,
                                float* z, void* stream) {

@@ -116,6 +116,8 @@ WORKLOADS = {
     "c2": Workload("c2", N=8192, d=4096, E=16, I=688, K=4, T=8, P=4, n_calib=8192),
     "c3": Workload("c3", N=16384, d=2048, E=60, I=1408, K=4, T=16, P=4, I_s=5632, n_calib=16384),
     "c4": Workload("c4", N=16384, d=2048, E=60, I=1408, K=4, T=16, P=4, I_s=5632, n_calib=16384, backward=False, skew=True),
+    # c3 shapes on a quarter of the tokens: the small case for profiler captures
+    "c3s": Workload("c3s", N=4096, d=2048, E=60, I=1408, K=4, T=16, P=4, I_s=5632, n_calib=4096),
     "c5": Workload("c5", N=65536, d=2048, E=60, I=1408, K=4, T=16, P=4, I_s=5632, n_calib=65536),
 }
 
