@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libc2r.so")
-SOURCES = ["route.cu", "permute.cu", "gemm_simt.cu", "gemm_tc.cu", "api.cu"]
+SOURCES = ["route.cu", "permute.cu", "gemm_simt.cu", "gemm_tc.cu", "gate_tc.cu", "api.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -126,7 +126,7 @@ extern "C" int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
     C2R_REQUIRE(b->wsg && b->z && b->Ws13p && b->Ws2 && b->ABs && b->Hs && b->Ys && b->s_counts && b->s_offsets,
                 C2R_ERR_INVALID_ARG);
   const int64_t R = permuted_rows(cfg);
-  C2R_TRY(c2r_gate_logits(cfg, b->X, b->Wg, shared ? b->wsg : nullptr, b->L, b->z, stream));
+  C2R_TRY(gate_logits_impl(cfg, b->X, b->Wg, shared ? b->wsg : nullptr, b->L, b->z, b->status, stream));
   C2R_TRY(c2r_route(cfg, b->L, b->mask, b->idx, b->w, nullptr, b->status, stream));
   C2R_TRY(c2r_permute(cfg, b->idx, b->expert_rank, b->X, b->counts, b->offsets, b->row_of_slot, b->slot_of_row, b->Xp,
                       b->status, b->ws, b->ws_bytes, stream));

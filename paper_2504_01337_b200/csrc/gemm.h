@@ -49,6 +49,14 @@ int tc_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* X
                   const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status,
                   cudaStream_t s);
 
+// Gate logits on the tensor cores (bf16 only).
+bool gate_tc_supported(const c2r_config* cfg);
+int gate_tc_launch(const c2r_config* cfg, const void* X, const void* Wg, const void* wsg, float* L, float* z,
+                   int32_t* status, cudaStream_t s);
+// c2r_gate_logits with a status word for the bounded waits of the tensor-core kernel.
+int gate_logits_impl(const c2r_config* cfg, const void* X, const void* Wg, const void* wsg, float* L, float* z,
+                     int32_t* status, void* stream);
+
 size_t permute_ws_bytes(const c2r_config* cfg);
 size_t gate_bwd_ws_bytes(const c2r_config* cfg);
 

@@ -9,22 +9,16 @@
 // (tmem_full/tmem_empty) between MMA and epilogue, so the epilogue of tile i overlaps the MMAs of
 // tile i+1.  Every wait is bounded: on expiry the kernel raises C2R_STATUS_WAIT_TIMEOUT in the
 // status word, all roles leave their loops, TMEM is released and the kernel returns.
-#include <cuda.h>
-
-#include "c2r_common.cuh"
 #include "gemm.h"
+#include "tc_common.cuh"
 
 namespace c2r {
 
-constexpr int BM = 128;
-constexpr int BK = 64;          // 64 bf16 = one 128-byte swizzle row
-constexpr int UMMA_K = 16;
 constexpr int STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * BK * 2;        // 16 KB
 constexpr int B_STAGE_BYTES_MAX = 256 * BK * 2;   // 32 KB
 constexpr int TC_THREADS = 192;
 constexpr int TMEM_COLS = 512;
-constexpr uint32_t WAIT_LIMIT = 1u << 24;         // try_wait polls before a wait gives up
 
 struct TcParams {
   int mode;        // TC_ROWS / TC_WGRAD
@@ -46,95 +40,6 @@ struct TcParams {
   void* H;         // TC_EPI_SWIGLU_FWD: H output
   int32_t* status;
 };
-
-// ---- PTX wrappers ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait; false = gave up (or another role already aborted).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 1023u) == 1023u && *abort_flag) return false;
-  }
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-      "l"(map), "r"(bar), "r"(x), "r"(y)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
-      "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
-      : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-      "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor (sm_100 format): 128-byte swizzle, 16-byte units.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= (uint64_t)1 << 46;  // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;  // SWIZZLE_128B
-  return d;
-}
-
-// bf16 x bf16 -> f32 instruction descriptor, M = 128.
-__device__ __forceinline__ uint32_t instr_desc(int n, bool a_mn, bool b_mn) {
-  uint32_t d = 0;
-  d |= 1u << 4;                     // D format f32
-  d |= 1u << 7;                     // A format bf16
-  d |= 1u << 10;                    // B format bf16
-  d |= (a_mn ? 1u : 0u) << 15;      // A major: 0 = K, 1 = MN
-  d |= (b_mn ? 1u : 0u) << 16;      // B major
-  d |= (uint32_t)(n >> 3) << 17;    // N / 8
-  d |= (uint32_t)(BM >> 4) << 24;   // M / 16
-  return d;
-}
 
 struct TileInfo {
   int expert;   // group
@@ -344,14 +249,80 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       int n_mma, w;
       n_geometry<BN>(p, ti.jn, n_mma, w);
       const bool have_acc = ti.kblocks > 0;
-      if (have_acc) {
-        if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-      }
       const int row_in_tile = 32 * q + lane;
       const uint32_t taddr_row = tmem_base + acc * 256 + ((uint32_t)(32 * q) << 16);
       const int mrow = ti.m0 + row_in_tile;
       const bool row_ok = (p.mode == TC_ROWS) ? (mrow < p.R) : (mrow < p.Mout);
+      if (p.epi == TC_EPI_SWIGLU_BWD) {
+        // The saved (A, B) do not depend on the accumulator: four 16-column chunks of both are
+        // requested at once (and the first batch before the accumulator is awaited), so a tile
+        // pays two global-memory round trips instead of one per chunk.
+        const __nv_bfloat16* ab = (const __nv_bfloat16*)p.AB + (long long)mrow * 2 * p.I + 256 * ti.jn;
+        __nv_bfloat16* dab = (__nv_bfloat16*)p.C + (long long)mrow * 2 * p.I + 256 * ti.jn;
+        bool waited = !have_acc;
+        for (int c0 = 0; c0 < w; c0 += 64) {
+          uint4 qa[4][2], qb[4][2];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int c = c0 + 16 * j;
+            if (row_ok && c < w) {
+              qa[j][0] = reinterpret_cast<const uint4*>(ab + c)[0];
+              qa[j][1] = reinterpret_cast<const uint4*>(ab + c)[1];
+              qb[j][0] = reinterpret_cast<const uint4*>(ab + w + c)[0];
+              qb[j][1] = reinterpret_cast<const uint4*>(ab + w + c)[1];
+            } else {
+              qa[j][0] = qa[j][1] = qb[j][0] = qb[j][1] = make_uint4(0, 0, 0, 0);
+            }
+          }
+          if (!waited) {
+            if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            waited = true;
+          }
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int c = c0 + 16 * j;
+            if (c >= w) break;  // warp-uniform
+            uint32_t r0[16];
+            float v0[16];
+            if (have_acc) {
+              tc_ld16(taddr_row + c, r0);
+              tc_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 16; ++i) v0[i] = __uint_as_float(r0[i]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 16; ++i) v0[i] = 0.f;
+            }
+            if (!row_ok) continue;
+            const uint32_t ua[8] = {qa[j][0].x, qa[j][0].y, qa[j][0].z, qa[j][0].w, qa[j][1].x, qa[j][1].y, qa[j][1].z, qa[j][1].w};
+            const uint32_t ub[8] = {qb[j][0].x, qb[j][0].y, qb[j][0].z, qb[j][0].w, qb[j][1].x, qb[j][1].y, qb[j][1].z, qb[j][1].w};
+            float da[16], db[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float a = __uint_as_float((i & 1) ? (ua[i >> 1] & 0xFFFF0000u) : (ua[i >> 1] << 16));
+              const float b = __uint_as_float((i & 1) ? (ub[i >> 1] & 0xFFFF0000u) : (ub[i >> 1] << 16));
+              const float s = 1.0f / (1.0f + __expf(-a));
+              da[i] = v0[i] * b * (s * (1.0f + a * (1.0f - s)));
+              db[i] = v0[i] * (a * s);
+            }
+            store_bf16x16(dab + c, da);
+            store_bf16x16(dab + w + c, db);
+          }
+        }
+        if (!ok) break;
+        if (have_acc) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        continue;
+      }
+      if (have_acc) {
+        if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+      }
       for (int c = 0; c < w; c += 16) {
         uint32_t r0[16], r1[16];
         float v0[16], v1[16];
@@ -375,21 +346,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 16; ++i) h[i] = v0[i] / (1.0f + __expf(-v0[i])) * v1[i];
           store_bf16x16((__nv_bfloat16*)p.H + (long long)mrow * p.I + 128 * ti.jn + c, h);
-        } else if (p.epi == TC_EPI_SWIGLU_BWD) {
-          const int pg = 256 * ti.jn + c, pu = pg + w;
-          const __nv_bfloat16* ab = (const __nv_bfloat16*)p.AB + (long long)mrow * 2 * p.I;
-          __nv_bfloat16* dab = (__nv_bfloat16*)p.C + (long long)mrow * 2 * p.I;
-          float a[16], b[16], da[16], db[16];
-          load_bf16x16(ab + pg, a);
-          load_bf16x16(ab + pu, b);
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float s = 1.0f / (1.0f + __expf(-a[i]));
-            da[i] = v0[i] * b[i] * (s * (1.0f + a[i] * (1.0f - s)));
-            db[i] = v0[i] * (a[i] * s);
-          }
-          store_bf16x16(dab + pg, da);
-          store_bf16x16(dab + pu, db);
         } else if (p.epi == TC_EPI_F32) {
           float* o = (float*)p.C + (long long)mrow * p.ldc + BN * ti.jn + c;
 #pragma unroll
@@ -427,48 +383,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn get_encode() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-  }
-  return fn;
-}
-
-// bf16 tensor map over a row-major array viewed as [d2][d1][d0] (d0 contiguous), box {b0, b1, 1}, 128-byte swizzle.
-static int make_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2, uint32_t b0, uint32_t b1) {
-  EncodeTiledFn enc = get_encode();
-  if (!enc) return C2R_ERR_CUDA;
-  cuuint64_t dims[3] = {d0, d1, d2};
-  cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
-  cuuint32_t box[3] = {b0, b1, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  const cuuint32_t rank = d2 > 0 ? 3 : 2;
-  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) { g_last_cuda_error = (int)cudaErrorInvalidValue; return C2R_ERR_CUDA; }
-  return C2R_OK;
-}
-
-static int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      n = 148;
-  }
-  return n;
-}
-
 template <bool A_MN, bool B_MN, int BN>
 static int launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, cudaStream_t s) {
   constexpr int smem = STAGES * (A_STAGE_BYTES + BN * BK * 2) + 1024;

@@ -2,6 +2,7 @@
 // Integer outputs are exact and independent of scheduling (integer atomics only where the
 // result does not depend on their order).
 #include "c2r_common.cuh"
+#include "gemm.h"
 
 namespace c2r {
 
@@ -264,14 +265,16 @@ extern "C" int c2r_last_cuda_error(void) { return g_last_cuda_error; }
 
 extern "C" uint64_t c2r_launch_count(void) { return __atomic_load_n(&g_launch_count, __ATOMIC_RELAXED); }
 
-extern "C" int c2r_gate_logits(const c2r_config* cfg, const void* X, const void* Wg, const void* wsg, float* L,
-                               float* z, void* stream) {
+int c2r::gate_logits_impl(const c2r_config* cfg, const void* X, const void* Wg, const void* wsg, float* L, float* z,
+                          int32_t* status, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   C2R_REQUIRE(X && Wg && L, C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(!wsg || z, C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(cfg->E + (wsg ? 1 : 0) <= GL_COLS, C2R_ERR_UNSUPPORTED_SHAPE);
   if (cfg->N == 0) return C2R_OK;
+  const bool aligned = (((uintptr_t)X | (uintptr_t)Wg | (uintptr_t)wsg | (uintptr_t)L) & 15u) == 0;
+  if (aligned && gate_tc_supported(cfg)) return gate_tc_launch(cfg, X, Wg, wsg, L, z, status, as_stream(stream));
   dim3 grid((cfg->N + GL_TM - 1) / GL_TM);
   if (cfg->dtype == C2R_BF16)
     gate_logits_kernel<__nv_bfloat16><<<grid, 256, 0, as_stream(stream)>>>(
@@ -281,6 +284,11 @@ extern "C" int c2r_gate_logits(const c2r_config* cfg, const void* X, const void*
                                                                    (const float*)wsg, L, z, cfg->N, cfg->d, cfg->E);
   C2R_LAUNCH_CHECK();
   return C2R_OK;
+}
+
+extern "C" int c2r_gate_logits(const c2r_config* cfg, const void* X, const void* Wg, const void* wsg, float* L,
+                               float* z, void* stream) {
+  return gate_logits_impl(cfg, X, Wg, wsg, L, z, nullptr, stream);
 }
 
 extern "C" int c2r_route(const c2r_config* cfg, const float* L, const uint64_t* mask, int32_t* idx, float* w, float* p,

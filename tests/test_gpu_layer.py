@@ -27,18 +27,22 @@ def _close(bf16, stored_bf16=True):
 
 
 @pytest.mark.parametrize("bf16", [False, True])
-def test_gate_logits(bf16):
+@pytest.mark.parametrize("N,d,E,shared", [(1000, 256, 60, True), (129, 200, 8, False), (4096, 2048, 33, True),
+                                          (1, 64, 5, True), (300, 1032, 64, False), (20000, 128, 63, True)])
+def test_gate_logits(bf16, N, d, E, shared):
+    """Eq. 1 logits; the bf16 cases run the tcgen05 streaming kernel (several tiles per CTA at N=20000,
+    ragged token and contraction tails, fewer experts than the 64-row weight box)."""
     b = B()
-    N, d, E = 1000, 256, 60
     X = G.normal(1, G.S_X, (N, d)); Wg = G.normal(1, G.S_WG, (E, d), 0.02); wsg = G.normal(1, G.S_WSG, (d,), 0.02)
     if bf16:
         X, Wg, wsg = G.round_bf16(X), G.round_bf16(Wg), G.round_bf16(wsg)
     dt = torch.bfloat16 if bf16 else None
-    cfg = b.make_config(N, d, E, 16, 4, 8, 1, 16, b.BF16 if bf16 else b.F32, 1)
-    L = torch.zeros((N, E), device="cuda"); z = torch.zeros((N,), device="cuda")
-    b.gate_logits(cfg, dev(X, dt), dev(Wg, dt), dev(wsg, dt), L, z)
+    cfg = b.make_config(N, d, E, 16, min(4, E), min(8, E - 1), 1, 16 if shared else 0, b.BF16 if bf16 else b.F32, 1)
+    L = torch.full((N, E), 7.0, device="cuda"); z = torch.full((N,), 7.0, device="cuda")
+    b.gate_logits(cfg, dev(X, dt), dev(Wg, dt), dev(wsg, dt) if shared else None, L, z if shared else None)
     assert_close_abs(host(L), O.gate_logits(X, Wg), 1e-4, "L")
-    assert_close_abs(host(z), X.astype(np.float64) @ wsg.astype(np.float64), 1e-4, "z")
+    if shared:
+        assert_close_abs(host(z), X.astype(np.float64) @ wsg.astype(np.float64), 1e-4, "z")
 
 
 def test_c1_layer_forward_fp32():
