@@ -11,7 +11,7 @@
 // Warp roles (320 threads per CTA): warp 0 = TMA producer (both CTAs, each for its own halves),
 // warp 1 = MMA issuer (even CTA only; owns the TMEM allocation in both), warps 2..9 = epilogue
 // (TMEM -> registers -> global, fused SwiGLU forms; two warps per TMEM lane quarter).
-// Pipelines: 6 shared-memory stages (full barrier in the even CTA counts both CTAs' bytes; the
+// Pipelines: 5 shared-memory stages (full barrier in the even CTA counts both CTAs' bytes; the
 // MMA's commit frees the stage in both CTAs) and two TMEM accumulators of 256 columns, so the
 // epilogue of tile i overlaps the MMAs of tile i+1.  Every wait is bounded: on expiry the kernel
 // raises C2R_STATUS_WAIT_TIMEOUT in the status word, the roles leave their loops, both CTAs meet
@@ -21,12 +21,14 @@
 
 namespace c2r {
 
-constexpr int STAGES = 6;
+constexpr int STAGES = 5;
 constexpr int HALF_BYTES = 128 * BK * 2;          // one CTA's share of either operand per stage: 16 KB
 constexpr int STAGE_BYTES = 2 * HALF_BYTES;       // A half + B half
 constexpr int TC_THREADS = 320;
 constexpr int EPI_WARPS = 8;
 constexpr int TMEM_COLS = 512;
+constexpr int STG_BYTES = 32 * 128;                // a warp's staging tile: 32 rows x 128 bytes
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * 2 * STG_BYTES + 1024;
 constexpr int TILE_M = 256;                       // rows of a pair tile (128 per CTA)
 constexpr int TILE_N = 256;                       // widest MMA-N
 
@@ -126,6 +128,52 @@ __device__ __forceinline__ void unpack_bf16x16(const uint4& a, const uint4& b, f
 }
 __device__ __forceinline__ void load_bf16x16(const __nv_bfloat16* src, float* v) {
   unpack_bf16x16(reinterpret_cast<const uint4*>(src)[0], reinterpret_cast<const uint4*>(src)[1], v);
+}
+
+__device__ __forceinline__ uint4 pack_bf16x8(const float* v) {
+  return make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+}
+
+// ---- warp-private staging tiles ---------------------------------------------------------------
+// 32 rows x 128 bytes.  The 16-byte chunks of a row are permuted by (chunk ^ (row & 7)), which
+// keeps both access patterns free of bank conflicts: "row per lane" (what a TMEM load gives a
+// thread) and "row contiguous" (8 lanes cover the 128 bytes of one row, 4 rows per instruction:
+// the coalesced shape for global memory).
+__device__ __forceinline__ uint32_t stg_addr(uint32_t buf, int row, int chunk) {
+  return buf + row * 128 + ((chunk ^ (row & 7)) << 4);
+}
+__device__ __forceinline__ void sts128(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+// Staging tile -> global rows [0, rows_valid) x bytes [0, valid_bytes) starting at g (row pitch in bytes).
+__device__ __forceinline__ void stage_to_global(uint32_t buf, uint8_t* g, long long pitch, int rows_valid, int valid_bytes,
+                                                int lane) {
+  const int chunk = lane & 7, sub = lane >> 3;
+  if (16 * chunk >= valid_bytes) return;
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int row = 4 * it + sub;
+    if (row < rows_valid) *reinterpret_cast<uint4*>(g + row * pitch + 16 * chunk) = lds128(stg_addr(buf, row, chunk));
+  }
+}
+// Global -> staging tile, same shape; all loads are issued before the first store to shared memory.
+__device__ __forceinline__ void global_to_stage(uint32_t buf, const uint8_t* g, long long pitch, int rows_valid,
+                                                int valid_bytes, int lane) {
+  const int chunk = lane & 7, sub = lane >> 3;
+  if (16 * chunk >= valid_bytes) return;
+  uint4 v[8];
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int row = 4 * it + sub;
+    v[it] = (row < rows_valid) ? *reinterpret_cast<const uint4*>(g + row * pitch + 16 * chunk) : make_uint4(0, 0, 0, 0);
+  }
+#pragma unroll
+  for (int it = 0; it < 8; ++it) sts128(stg_addr(buf, 4 * it + sub, chunk), v[it]);
 }
 
 // A_MN / B_MN: operand is MN-major in global memory (the contraction index is the row index).
@@ -260,8 +308,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
   } else {
     // ------------------------------- epilogue (8 warps) -------------------------------------
-    const int q = warp & 3;           // TMEM lane quarter this warp may read
-    const int hsel = (warp - 2) >> 2;  // which of the two warps of that quarter: takes every other 16-column chunk
+    // TMEM hands every thread one accumulator row, which is the worst shape for global memory (32
+    // rows per access).  Each warp therefore passes its 32 x 128-byte pieces through a private
+    // staging tile in shared memory and moves them to / from global memory row-contiguously.
+    const int q = warp & 3;            // TMEM lane quarter this warp may read
+    const int hsel = (warp - 2) >> 2;  // which of the two warps of that quarter: takes every other column group
+    const uint32_t buf0 = smem_base + STAGES * STAGE_BYTES + (warp - 2) * (2 * STG_BYTES), buf1 = buf0 + STG_BYTES;
     const uint32_t tempty_mma0 = map_to_cta(tempty0, 0);
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
@@ -272,70 +324,60 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       n_geometry(p, ti.jn, n_mma, w, brow0);
       const bool have_acc = ti.kblocks > 0;
       const uint32_t taddr_row = tmem_base + acc * TILE_N + ((uint32_t)(32 * q) << 16);
-      const int mrow = ti.m0 + BM * (int)rank + 32 * q + lane;
-      const bool row_ok = mrow < ti.m_end;
-      const int n_chunks = w >> 4;
+      const int row0 = ti.m0 + BM * (int)rank + 32 * q;  // first of this warp's 32 rows
+      const int rows_valid = max(0, min(32, ti.m_end - row0));
+      const long long mrow = row0 + lane;
       bool waited = !have_acc;
       if (p.epi == TC_EPI_SWIGLU_BWD) {
-        // dA = dH * B * silu'(A), dB = dH * silu(A).  The saved (A, B) do not depend on the
-        // accumulator: up to four chunks of both are requested at once, the first batch before
-        // the accumulator is awaited.
-        const __nv_bfloat16* ab = (const __nv_bfloat16*)p.AB + (long long)mrow * 2 * p.I;
-        __nv_bfloat16* dab = (__nv_bfloat16*)p.C + (long long)mrow * 2 * p.I;
-        for (int ci0 = hsel; ci0 < n_chunks && ok; ci0 += 8) {
-          uint4 qa[4][2], qb[4][2];
-          int col_a[4], col_b[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int ci = ci0 + 2 * j;
-            const int hc = TILE_N * ti.jn + 16 * ci;  // H column of the chunk
-            const int blk = hc >> 7;                  // 128-channel block of the packed (A | B) layout
-            const int wj = min(128, p.I - 128 * blk);
-            col_a[j] = 256 * blk + (hc & 127);
-            col_b[j] = col_a[j] + wj;
-            if (row_ok && ci < n_chunks) {
-              qa[j][0] = reinterpret_cast<const uint4*>(ab + col_a[j])[0];
-              qa[j][1] = reinterpret_cast<const uint4*>(ab + col_a[j])[1];
-              qb[j][0] = reinterpret_cast<const uint4*>(ab + col_b[j])[0];
-              qb[j][1] = reinterpret_cast<const uint4*>(ab + col_b[j])[1];
-            } else {
-              qa[j][0] = qa[j][1] = qb[j][0] = qb[j][1] = make_uint4(0, 0, 0, 0);
-            }
-          }
+        // dA = dH * B * silu'(A), dB = dH * silu(A) on groups of 64 H columns.  The saved (A, B) do
+        // not depend on the accumulator, so the first group's loads are issued before it is awaited.
+        const int n_groups = (w + 63) >> 6;
+        for (int g = hsel; g < n_groups; g += 2) {
+          const int hc0 = TILE_N * ti.jn + 64 * g;  // first H column of the group; a group never leaves its
+          const int blk = hc0 >> 7;                 // 128-channel block of the packed (A | B) layout
+          const int col_a = 256 * blk + (hc0 & 127);
+          const int col_b = col_a + min(128, p.I - 128 * blk);
+          const int vbytes = 2 * min(64, w - 64 * g);
+          const long long pitch = 4ll * p.I;  // bytes per row of AB / dAB
+          const uint8_t* ga = (const uint8_t*)p.AB + row0 * pitch;
+          uint8_t* go = (uint8_t*)p.C + row0 * pitch;
+          global_to_stage(buf0, ga + 2 * col_a, pitch, rows_valid, vbytes, lane);
+          global_to_stage(buf1, ga + 2 * col_b, pitch, rows_valid, vbytes, lane);
+          __syncwarp();
           if (!waited) {
             if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             waited = true;
           }
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int ci = ci0 + 2 * j;
-            if (ci >= n_chunks) break;  // warp-uniform
+          for (int pc = 0; pc < 4; ++pc) {
+            if (32 * pc >= vbytes) break;  // warp-uniform
             uint32_t r0[16];
-            float v0[16];
+            float v0[16], a[16], b[16], da[16], db[16];
             if (have_acc) {
-              tc_ld16(taddr_row + 16 * ci, r0);
+              tc_ld16(taddr_row + 64 * g + 16 * pc, r0);
               tc_ld_wait();
-#pragma unroll
-              for (int i = 0; i < 16; ++i) v0[i] = __uint_as_float(r0[i]);
-            } else {
-#pragma unroll
-              for (int i = 0; i < 16; ++i) v0[i] = 0.f;
             }
-            if (!row_ok) continue;
-            float a[16], b[16], da[16], db[16];
-            unpack_bf16x16(qa[j][0], qa[j][1], a);
-            unpack_bf16x16(qb[j][0], qb[j][1], b);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v0[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
+            const uint32_t sa0 = stg_addr(buf0, lane, 2 * pc), sa1 = stg_addr(buf0, lane, 2 * pc + 1);
+            const uint32_t sb0 = stg_addr(buf1, lane, 2 * pc), sb1 = stg_addr(buf1, lane, 2 * pc + 1);
+            unpack_bf16x16(lds128(sa0), lds128(sa1), a);
+            unpack_bf16x16(lds128(sb0), lds128(sb1), b);
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
               const float s = sigmoid_fast(a[i]);
-              const float as = a[i] * s;                  // silu(a)
-              da[i] = v0[i] * b[i] * (s + as - as * s);   // silu'(a) = s (1 + a (1 - s))
+              const float as = a[i] * s;                 // silu(a)
+              da[i] = v0[i] * b[i] * (s + as - as * s);  // silu'(a) = s (1 + a (1 - s))
               db[i] = v0[i] * as;
             }
-            store_bf16x16(dab + col_a[j], da);
-            store_bf16x16(dab + col_b[j], db);
+            sts128(sa0, pack_bf16x8(da)); sts128(sa1, pack_bf16x8(da + 8));
+            sts128(sb0, pack_bf16x8(db)); sts128(sb1, pack_bf16x8(db + 8));
           }
+          __syncwarp();
+          stage_to_global(buf0, go + 2 * col_a, pitch, rows_valid, vbytes, lane);
+          stage_to_global(buf1, go + 2 * col_b, pitch, rows_valid, vbytes, lane);
+          __syncwarp();
         }
         if (!ok) break;
       }
@@ -343,49 +385,110 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
         tc_fence_after();
       }
-      if (p.epi != TC_EPI_SWIGLU_BWD) {
-        for (int ci = hsel; ci < n_chunks; ci += 2) {
-          const int c = 16 * ci;
-          uint32_t r0[16], r1[16];
-          float v0[16], v1[16];
-          if (have_acc) {
-            tc_ld16(taddr_row + c, r0);
-            if (p.epi == TC_EPI_SWIGLU_FWD) tc_ld16(taddr_row + w + c, r1);
-            tc_ld_wait();
+      if (p.epi == TC_EPI_SWIGLU_FWD) {
+        // accumulator columns [0,w) = gate (A), [w,2w) = up (B): store both packed and H = silu(A) * B
+        const int n_groups = (w + 63) >> 6;
+        for (int g = hsel; g < n_groups; g += 2) {
+          const int c = 64 * g;
+          const int vbytes = 2 * min(64, w - c);
+          uint4 up[8];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) { v0[i] = __uint_as_float(r0[i]); v1[i] = __uint_as_float(r1[i]); }
-          } else {
+          for (int pc = 0; pc < 4; ++pc) {
+            if (32 * pc >= vbytes) break;
+            uint32_t r0[16], r1[16];
+            float v0[16], v1[16], h[16];
+            if (have_acc) {
+              tc_ld16(taddr_row + c + 16 * pc, r0);
+              tc_ld16(taddr_row + w + c + 16 * pc, r1);
+              tc_ld_wait();
+            }
 #pragma unroll
-            for (int i = 0; i < 16; ++i) { v0[i] = 0.f; v1[i] = 0.f; }
+            for (int i = 0; i < 16; ++i) {
+              v0[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
+              v1[i] = have_acc ? __uint_as_float(r1[i]) : 0.f;
+              h[i] = v0[i] * sigmoid_fast(v0[i]) * v1[i];
+            }
+            sts128(stg_addr(buf0, lane, 2 * pc), pack_bf16x8(v0)); sts128(stg_addr(buf0, lane, 2 * pc + 1), pack_bf16x8(v0 + 8));
+            sts128(stg_addr(buf1, lane, 2 * pc), pack_bf16x8(h)); sts128(stg_addr(buf1, lane, 2 * pc + 1), pack_bf16x8(h + 8));
+            up[2 * pc] = pack_bf16x8(v1); up[2 * pc + 1] = pack_bf16x8(v1 + 8);
           }
-          if (!row_ok) continue;
-          if (p.epi == TC_EPI_SWIGLU_FWD) {
-            // accumulator columns [0,w) = gate (A), [w,2w) = up (B): store both packed and H = silu(A) * B
-            const int pg = 256 * ti.jn + c, pu = pg + w;
-            __nv_bfloat16* ab = (__nv_bfloat16*)p.C + (long long)mrow * 2 * p.I;
-            store_bf16x16(ab + pg, v0);
-            store_bf16x16(ab + pu, v1);
-            float h[16];
+          __syncwarp();
+          uint8_t* gab = (uint8_t*)p.C + row0 * (4ll * p.I) + 2 * (256 * ti.jn + c);
+          stage_to_global(buf0, gab, 4ll * p.I, rows_valid, vbytes, lane);
+          stage_to_global(buf1, (uint8_t*)p.H + row0 * (2ll * p.I) + 2 * (128 * ti.jn + c), 2ll * p.I, rows_valid, vbytes, lane);
+          __syncwarp();
 #pragma unroll
-            for (int i = 0; i < 16; ++i) h[i] = v0[i] * sigmoid_fast(v0[i]) * v1[i];
-            store_bf16x16((__nv_bfloat16*)p.H + (long long)mrow * p.I + 128 * ti.jn + c, h);
-          } else if (p.epi == TC_EPI_F32) {
-            float* o = (float*)p.C + (long long)mrow * p.ldc + TILE_N * ti.jn + c;
+          for (int pc = 0; pc < 4; ++pc) {
+            if (32 * pc >= vbytes) break;
+            sts128(stg_addr(buf0, lane, 2 * pc), up[2 * pc]); sts128(stg_addr(buf0, lane, 2 * pc + 1), up[2 * pc + 1]);
+          }
+          __syncwarp();
+          stage_to_global(buf0, gab + 2 * w, 4ll * p.I, rows_valid, vbytes, lane);
+          __syncwarp();
+        }
+      } else if (p.epi == TC_EPI_F32) {
+        const int n_groups = (w + 31) >> 5;  // 32 fp32 columns = 128 bytes
+        for (int g = hsel; g < n_groups; g += 2) {
+          const int c = 32 * g;
+          const int vbytes = 4 * min(32, w - c);
+          const uint32_t buf = (g & 2) ? buf1 : buf0;  // alternate tiles: the next group's writes need not wait
+#pragma unroll
+          for (int pc = 0; pc < 2; ++pc) {
+            if (64 * pc >= vbytes) break;
+            uint32_t r0[16];
+            if (have_acc) {
+              tc_ld16(taddr_row + c + 16 * pc, r0);
+              tc_ld_wait();
+            }
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              reinterpret_cast<float4*>(o)[i] = make_float4(v0[4 * i], v0[4 * i + 1], v0[4 * i + 2], v0[4 * i + 3]);
-          } else {  // TC_EPI_WGRAD_BF16
-            __nv_bfloat16* o =
-                (__nv_bfloat16*)p.C + (long long)ti.expert * p.sC + (long long)mrow * p.ldc + TILE_N * ti.jn + c;
-            if (p.accumulate) {
-              float old[16];
-              load_bf16x16(o, old);
+              sts128(stg_addr(buf, lane, 4 * pc + i),
+                     have_acc ? make_uint4(r0[4 * i], r0[4 * i + 1], r0[4 * i + 2], r0[4 * i + 3]) : make_uint4(0, 0, 0, 0));
+          }
+          __syncwarp();
+          stage_to_global(buf, (uint8_t*)p.C + row0 * (4 * p.ldc) + 4ll * (TILE_N * ti.jn + c), 4 * p.ldc, rows_valid, vbytes,
+                          lane);
+        }
+        __syncwarp();
+      } else if (p.epi == TC_EPI_WGRAD_BF16) {
+        const int n_groups = (w + 63) >> 6;
+        for (int g = hsel; g < n_groups; g += 2) {
+          const int c = 64 * g;
+          const int vbytes = 2 * min(64, w - c);
+          __nv_bfloat16* orow = (__nv_bfloat16*)p.C + (long long)ti.expert * p.sC + mrow * p.ldc + TILE_N * ti.jn + c;
+          const uint32_t buf = (g & 2) ? buf1 : buf0;
 #pragma unroll
-              for (int i = 0; i < 16; ++i) v0[i] += old[i];
+          for (int pc = 0; pc < 4; ++pc) {
+            if (32 * pc >= vbytes) break;
+            uint32_t r0[16];
+            float v0[16];
+            if (have_acc) {
+              tc_ld16(taddr_row + c + 16 * pc, r0);
+              tc_ld_wait();
             }
-            store_bf16x16(o, v0);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v0[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
+            if (p.accumulate) {  // read-modify-write in fp32 straight on the thread's own row
+              if (lane < rows_valid) {
+                float old[16];
+                load_bf16x16(orow + 16 * pc, old);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) v0[i] += old[i];
+                store_bf16x16(orow + 16 * pc, v0);
+              }
+            } else {
+              sts128(stg_addr(buf, lane, 2 * pc), pack_bf16x8(v0));
+              sts128(stg_addr(buf, lane, 2 * pc + 1), pack_bf16x8(v0 + 8));
+            }
+          }
+          if (!p.accumulate) {
+            __syncwarp();
+            stage_to_global(buf, (uint8_t*)((__nv_bfloat16*)p.C + (long long)ti.expert * p.sC + (long long)row0 * p.ldc +
+                                            TILE_N * ti.jn + c),
+                            2 * p.ldc, rows_valid, vbytes, lane);
           }
         }
+        __syncwarp();
       }
       if (have_acc) {
         tc_fence_before();
@@ -412,7 +515,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 template <bool A_MN, bool B_MN>
 static int launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, cudaStream_t s) {
-  constexpr int smem = STAGES * STAGE_BYTES + 1024;
+  constexpr int smem = SMEM_BYTES;
   constexpr int MAX_DEV = 64;
   static int grid_of_device[MAX_DEV] = {};  // CTAs of the persistent grid (2 per co-resident pair), per device
   int dev = 0;
