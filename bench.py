@@ -106,9 +106,10 @@ class ClockSampler:
                 "samples": len(sm), "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons)}
 
 
-def build_layer(wl, device, profile=True):
+def build_layer(wl, device, profile=True, keep=False):
     """Seeded synthetic layer of workload `wl` on `device`, routed with collaborator sets profiled
-    from a calibration batch by the library itself (Eq. 2 / Eq. 4) and placed by co-activation."""
+    from a calibration batch by the library itself (Eq. 2 / Eq. 4) and placed by co-activation.
+    keep=True also returns the calibration state (device logits, routing, C, I_T, placement)."""
     import torch
     from paper_2504_01337_b200 import binding as B
     from paper_2504_01337_b200 import inputs as G
@@ -138,6 +139,8 @@ def build_layer(wl, device, profile=True):
     rank = torch.zeros(wl.E, dtype=torch.int32)
     B.place_experts(cal, Cm.cpu(), 0, part, rank)
     lay.set_routing(mask=mask, expert_rank=rank.to(device), part=part.to(device))
+    if keep:
+        return lay, dict(L=Lc, idx=idxc, C=Cm, I_T=I_T, mask=mask, part=part, rank=rank)
     del Xc, Lc
     return lay
 

@@ -163,8 +163,9 @@ int c2r_unpack_weights(const c2r_config* cfg, int n_experts, int I, const void* 
  * For each expert e on rows [offsets[e], offsets[e]+counts[e]) of Xp:
  *   A = Xp W1_e^T, B = Xp W3_e^T, H = silu(A) * B, Yp = H W2_e^T.
  * Xp [R,d] T; counts [n_experts], offsets [n_experts+1] int32 (device); W13p packed (above);
- * W2 [n_experts, d, I] T.  out: AB [R, 2I] T (A and B in the packed column layout, kept for the
- * backward pass), H [R,I] T, Yp [R,d] float.
+ * W2 [n_experts, d, I] T.  out: AB [R, 2I] T (what the backward pass needs from A and B, in the
+ * packed column layout: the local derivatives dH/dA = B silu'(A) in the gate columns and
+ * dH/dB = silu(A) in the up columns), H [R,I] T, Yp [R,d] float.
  * R = rows of the buffers.  Padding rows of Xp must be zero.  n_experts = 1 with counts = {R},
  * offsets = {0,R} evaluates the dense shared expert.
  * bf16 runs on the tensor cores (tcgen05) when d % 16 == 0 and, for n_experts > 1, row_align is a

@@ -129,21 +129,23 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(SimtGemm g) {
         TC* o = C + (long long)m * g.ldc + n;
         if (g.accumulate) v += to_f32(*o);
         *o = from_f32<TC>(v);
-      } else if (g.epi == SIMT_EPI_SWIGLU_FWD) {  // v = A[r,n], acc2 = B[r,n]: keep both, H = silu(A) * B
+      } else if (g.epi == SIMT_EPI_SWIGLU_FWD) {
+        // v = A[r,n], acc2 = B[r,n]: H = silu(A) * B; the backward pass needs only the two local
+        // derivatives dH/dA = B silu'(A) and dH/dB = silu(A), which are what is kept (packed columns)
         const int pg = pack_col(n, g.I), pu = pg + pack_width(n, g.I);
         const float b = acc2[i][j];
-        T* ab = (T*)g.C + (long long)(r0 + m) * 2 * g.I;
-        ab[pg] = from_f32<T>(v);
-        ab[pu] = from_f32<T>(b);
-        ((T*)g.aux_out)[(long long)(r0 + m) * g.I + n] = from_f32<T>(v / (1.0f + expf(-v)) * b);
-      } else {  // SIMT_EPI_SWIGLU_BWD: v = dH[r, n]; read (A,B) and write (dA,dB) at the packed columns
+        const float sg = 1.0f / (1.0f + expf(-v));
+        const float as = v * sg;
+        T* sv = (T*)g.C + (long long)(r0 + m) * 2 * g.I;
+        sv[pg] = from_f32<T>(b * (sg + as - as * sg));
+        sv[pu] = from_f32<T>(as);
+        ((T*)g.aux_out)[(long long)(r0 + m) * g.I + n] = from_f32<T>(as * b);
+      } else {  // SIMT_EPI_SWIGLU_BWD: v = dH[r, n]; dA = dH * (dH/dA), dB = dH * (dH/dB) at the packed columns
         const int pg = pack_col(n, g.I), pu = pg + pack_width(n, g.I);
-        const T* ab = (const T*)g.aux + (long long)(r0 + m) * 2 * g.I;
+        const T* sv = (const T*)g.aux + (long long)(r0 + m) * 2 * g.I;
         T* dab = (T*)g.C + (long long)(r0 + m) * 2 * g.I;
-        const float a = to_f32(ab[pg]), b = to_f32(ab[pu]);
-        const float s = 1.0f / (1.0f + expf(-a));
-        dab[pg] = from_f32<T>(v * b * (s * (1.0f + a * (1.0f - s))));
-        dab[pu] = from_f32<T>(v * (a * s));
+        dab[pg] = from_f32<T>(v * to_f32(sv[pg]));
+        dab[pu] = from_f32<T>(v * to_f32(sv[pu]));
       }
     }
   }
@@ -166,7 +168,7 @@ int simt_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void*
   const int max_m = (int)R;
   SimtGemm g{};
   g.counts = counts; g.offsets = offsets; g.mode = SIMT_ROWS; g.I = I;
-  // A = Xp W1^T, B = Xp W3^T in one pass over Xp; epilogue stores (A, B) packed and H = silu(A) * B
+  // A = Xp W1^T, B = Xp W3^T in one pass over Xp; epilogue stores H = silu(A) * B and its two local derivatives
   g.epi = SIMT_EPI_SWIGLU_FWD; g.aux_out = H;
   g.A = Xp; g.sam = d; g.sak = 1; g.B = W13p; g.sbn = d; g.sbk = 1; g.sB = (long long)2 * I * d;
   g.C = AB; g.ldc = 2 * I; g.Ndim = I; g.Kdim = d;

@@ -161,17 +161,21 @@ __device__ __forceinline__ void stage_to_global(uint32_t buf, uint8_t* g, long l
     if (row < rows_valid) *reinterpret_cast<uint4*>(g + row * pitch + 16 * chunk) = lds128(stg_addr(buf, row, chunk));
   }
 }
-// Global -> staging tile, same shape; all loads are issued before the first store to shared memory.
-__device__ __forceinline__ void global_to_stage(uint32_t buf, const uint8_t* g, long long pitch, int rows_valid,
-                                                int valid_bytes, int lane) {
+// Global rows [0, rows_valid) x bytes [0, valid_bytes) -> registers in the row-contiguous shape
+// (v[it] = chunk (lane & 7) of row 4*it + (lane >> 3)); zeros elsewhere.
+__device__ __forceinline__ void global_rows_load(uint4 (&v)[8], const uint8_t* g, long long pitch, int rows_valid,
+                                                 int valid_bytes, int lane) {
   const int chunk = lane & 7, sub = lane >> 3;
-  if (16 * chunk >= valid_bytes) return;
-  uint4 v[8];
 #pragma unroll
   for (int it = 0; it < 8; ++it) {
     const int row = 4 * it + sub;
-    v[it] = (row < rows_valid) ? *reinterpret_cast<const uint4*>(g + row * pitch + 16 * chunk) : make_uint4(0, 0, 0, 0);
+    v[it] = (row < rows_valid && 16 * chunk < valid_bytes)
+                ? *reinterpret_cast<const uint4*>(g + row * pitch + 16 * chunk)
+                : make_uint4(0, 0, 0, 0);
   }
+}
+__device__ __forceinline__ void stage_rows_store(uint32_t buf, const uint4 (&v)[8], int lane) {
+  const int chunk = lane & 7, sub = lane >> 3;
 #pragma unroll
   for (int it = 0; it < 8; ++it) sts128(stg_addr(buf, 4 * it + sub, chunk), v[it]);
 }
@@ -329,8 +333,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const long long mrow = row0 + lane;
       bool waited = !have_acc;
       if (p.epi == TC_EPI_SWIGLU_BWD) {
-        // dA = dH * B * silu'(A), dB = dH * silu(A) on groups of 64 H columns.  The saved (A, B) do
-        // not depend on the accumulator, so the first group's loads are issued before it is awaited.
+        // dA = dH * (dH/dA), dB = dH * (dH/dB) on groups of 64 H columns; the forward pass saved both
+        // local derivatives.  They do not depend on the accumulator, so the first group's loads are
+        // issued before it is awaited.
         const int n_groups = (w + 63) >> 6;
         for (int g = hsel; g < n_groups; g += 2) {
           const int hc0 = TILE_N * ti.jn + 64 * g;  // first H column of the group; a group never leaves its
@@ -339,10 +344,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const int col_b = col_a + min(128, p.I - 128 * blk);
           const int vbytes = 2 * min(64, w - 64 * g);
           const long long pitch = 4ll * p.I;  // bytes per row of AB / dAB
-          const uint8_t* ga = (const uint8_t*)p.AB + row0 * pitch;
+          const uint8_t* gsrc = (const uint8_t*)p.AB + row0 * pitch;
           uint8_t* go = (uint8_t*)p.C + row0 * pitch;
-          global_to_stage(buf0, ga + 2 * col_a, pitch, rows_valid, vbytes, lane);
-          global_to_stage(buf1, ga + 2 * col_b, pitch, rows_valid, vbytes, lane);
+          uint4 in0[8], in1[8];  // both pieces are requested before either is parked in shared memory
+          global_rows_load(in0, gsrc + 2 * col_a, pitch, rows_valid, vbytes, lane);
+          global_rows_load(in1, gsrc + 2 * col_b, pitch, rows_valid, vbytes, lane);
+          stage_rows_store(buf0, in0, lane);
+          stage_rows_store(buf1, in1, lane);
           __syncwarp();
           if (!waited) {
             if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
@@ -353,7 +361,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int pc = 0; pc < 4; ++pc) {
             if (32 * pc >= vbytes) break;  // warp-uniform
             uint32_t r0[16];
-            float v0[16], a[16], b[16], da[16], db[16];
+            float v0[16], ga[16], gb[16], da[16], db[16];
             if (have_acc) {
               tc_ld16(taddr_row + 64 * g + 16 * pc, r0);
               tc_ld_wait();
@@ -362,15 +370,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int i = 0; i < 16; ++i) v0[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
             const uint32_t sa0 = stg_addr(buf0, lane, 2 * pc), sa1 = stg_addr(buf0, lane, 2 * pc + 1);
             const uint32_t sb0 = stg_addr(buf1, lane, 2 * pc), sb1 = stg_addr(buf1, lane, 2 * pc + 1);
-            unpack_bf16x16(lds128(sa0), lds128(sa1), a);
-            unpack_bf16x16(lds128(sb0), lds128(sb1), b);
+            unpack_bf16x16(lds128(sa0), lds128(sa1), ga);
+            unpack_bf16x16(lds128(sb0), lds128(sb1), gb);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float s = sigmoid_fast(a[i]);
-              const float as = a[i] * s;                 // silu(a)
-              da[i] = v0[i] * b[i] * (s + as - as * s);  // silu'(a) = s (1 + a (1 - s))
-              db[i] = v0[i] * as;
-            }
+            for (int i = 0; i < 16; ++i) { da[i] = v0[i] * ga[i]; db[i] = v0[i] * gb[i]; }
             sts128(sa0, pack_bf16x8(da)); sts128(sa1, pack_bf16x8(da + 8));
             sts128(sb0, pack_bf16x8(db)); sts128(sb1, pack_bf16x8(db + 8));
           }
@@ -386,7 +389,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tc_fence_after();
       }
       if (p.epi == TC_EPI_SWIGLU_FWD) {
-        // accumulator columns [0,w) = gate (A), [w,2w) = up (B): store both packed and H = silu(A) * B
+        // accumulator columns [0,w) = gate (A), [w,2w) = up (B): H = silu(A) * B, and for the backward pass
+        // its local derivatives dH/dA = B silu'(A) (gate columns of the packed buffer) and dH/dB = silu(A) (up columns)
         const int n_groups = (w + 63) >> 6;
         for (int g = hsel; g < n_groups; g += 2) {
           const int c = 64 * g;
@@ -396,7 +400,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           for (int pc = 0; pc < 4; ++pc) {
             if (32 * pc >= vbytes) break;
             uint32_t r0[16], r1[16];
-            float v0[16], v1[16], h[16];
+            float ga[16], gb[16], h[16];
             if (have_acc) {
               tc_ld16(taddr_row + c + 16 * pc, r0);
               tc_ld16(taddr_row + w + c + 16 * pc, r1);
@@ -404,13 +408,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-              v0[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
-              v1[i] = have_acc ? __uint_as_float(r1[i]) : 0.f;
-              h[i] = v0[i] * sigmoid_fast(v0[i]) * v1[i];
+              const float a = have_acc ? __uint_as_float(r0[i]) : 0.f;
+              const float b = have_acc ? __uint_as_float(r1[i]) : 0.f;
+              const float sg = sigmoid_fast(a);
+              const float as = a * sg;             // silu(a)
+              h[i] = as * b;
+              ga[i] = b * (sg + as - as * sg);     // b silu'(a), silu'(a) = s (1 + a (1 - s))
+              gb[i] = as;
             }
-            sts128(stg_addr(buf0, lane, 2 * pc), pack_bf16x8(v0)); sts128(stg_addr(buf0, lane, 2 * pc + 1), pack_bf16x8(v0 + 8));
+            sts128(stg_addr(buf0, lane, 2 * pc), pack_bf16x8(ga)); sts128(stg_addr(buf0, lane, 2 * pc + 1), pack_bf16x8(ga + 8));
             sts128(stg_addr(buf1, lane, 2 * pc), pack_bf16x8(h)); sts128(stg_addr(buf1, lane, 2 * pc + 1), pack_bf16x8(h + 8));
-            up[2 * pc] = pack_bf16x8(v1); up[2 * pc + 1] = pack_bf16x8(v1 + 8);
+            up[2 * pc] = pack_bf16x8(gb); up[2 * pc + 1] = pack_bf16x8(gb + 8);
           }
           __syncwarp();
           uint8_t* gab = (uint8_t*)p.C + row0 * (4ll * p.I) + 2 * (256 * ti.jn + c);

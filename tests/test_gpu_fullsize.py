@@ -1,0 +1,187 @@
+"""GPU parity at the full workload sizes, in the launch configuration bench.py times
+(bench.build_layer + c2r_train_step).
+
+What the oracle can afford in full it checks in full: every integer output (routing given the
+device's fp32 logits, counts, offsets, both row maps, the collaboration matrix and the refreshed
+Top-T sets, dispatch volume, placement).  Floating-point results are checked on samples the oracle
+computes one by one: the layer output and the input gradient of sampled tokens (each depends on
+its own token only), all three weight gradients of two whole experts, column slabs of the shared
+expert's weight gradients, and properties that hold at any size.
+"""
+import functools
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import c2r_oracle as O
+from paper_2504_01337_b200 import inputs as G
+from tests.util import assert_close_abs, assert_close_contraction, assert_close_elem, assert_close_rms
+
+pytestmark = pytest.mark.gpu
+
+
+@functools.lru_cache(maxsize=2)
+def _weights(seed, E, I, d, I_s, bf16):
+    wl = G.Workload("w", N=1, d=d, E=E, I=I, K=1, T=1, P=1, I_s=I_s, bf16=bf16, seed=seed)
+    return G.gate_weights(wl), G.expert_weights(wl), G.shared_weights(wl)
+
+
+def _sets_from_mask(mask_u64, E):
+    return [[j for j in range(E) if (int(m) >> j) & 1] for m in mask_u64]
+
+
+def _run(wl):
+    import bench
+    lay, cal = bench.build_layer(wl, "cuda:0", keep=True)
+    X, dY = G.hidden(wl), G.grad_out(wl)
+    lay.set_input(X, dY)
+    lay.train_step()
+    torch.cuda.synchronize()
+    assert int(lay.t["status"].item()) == 0
+    return lay, cal, X, dY
+
+
+def _check_calibration(wl, cal):
+    """Profiling on the calibration batch: conventional Top-K -> Eq. 2 -> Eq. 4 -> placement."""
+    Lc = cal["L"].cpu().numpy()
+    idx_ref, _ = O.topk_route(Lc, wl.K)
+    assert np.array_equal(cal["idx"].cpu().numpy(), idx_ref)
+    C_ref = O.collab_count(idx_ref, wl.E)
+    assert np.array_equal(cal["C"].cpu().numpy(), C_ref)
+    sets = O.collab_sets(C_ref, wl.T)
+    assert np.array_equal(cal["I_T"].cpu().numpy(), sets)
+    assert np.array_equal(cal["mask"].cpu().numpy().view(np.uint64), O.member_to_mask(O.sets_to_member(sets, wl.E)))
+    part_ref, rank_ref = O.place_experts(C_ref, wl.P)
+    assert np.array_equal(cal["part"].numpy(), part_ref) and np.array_equal(cal["rank"].numpy(), rank_ref)
+    return sets, part_ref, rank_ref
+
+
+def _check_integer_path(wl, lay, sets, part, rank):
+    """Everything downstream of the fp32 logits that is integer work, on the full batch."""
+    L = lay.host("L")
+    idx_ref, w_ref = O.c2r_route(L, sets, wl.K)
+    assert np.array_equal(lay.host("idx"), idx_ref)
+    assert_close_abs(lay.host("w"), w_ref, 1e-5, "w")
+    counts, offsets, ros, sor = O.permute_index(idx_ref, wl.E, rank, lay.cfg.row_align)
+    assert np.array_equal(lay.host("counts"), counts) and np.array_equal(lay.host("offsets"), offsets)
+    assert np.array_equal(lay.host("row_of_slot"), ros)
+    got_sor = lay.host("slot_of_row")
+    assert np.array_equal(got_sor[:sor.size], sor) and np.all(got_sor[sor.size:] == -1)
+    v = O.dispatch_volume(idx_ref, part, wl.P)
+    vol = lay.host("volume")
+    P = wl.P
+    assert vol[:4].tolist() == [v["naive"], v["dedup"], v["naive_x"], v["dedup_x"]]
+    assert np.array_equal(vol[4:4 + P * P].reshape(P, P), v["send_naive"])
+    assert np.array_equal(vol[4 + P * P:].reshape(P, P), v["send_dedup"])
+    C_live = O.collab_count(idx_ref, wl.E)
+    assert np.array_equal(lay.host("C"), C_live)
+    new_sets = O.collab_sets(C_live, wl.T)
+    assert np.array_equal(lay.host("I_T"), new_sets)
+    assert np.array_equal(lay.host("mask_next").view(np.uint64), O.member_to_mask(O.sets_to_member(new_sets, wl.E)))
+    return L, idx_ref, w_ref, counts, offsets, ros, sor
+
+
+def _dev_rows(t, rows):
+    """Rows `rows` (numpy int array) of device tensor t as float64 numpy."""
+    sel = t[torch.from_numpy(np.ascontiguousarray(rows)).to(t.device)]
+    return (sel.float() if sel.dtype == torch.bfloat16 else sel).cpu().numpy().astype(np.float64)
+
+
+def _check_sampled_tokens(wl, lay, X, dY, L, idx, sets, rank, n_sample):
+    """Forward and input-gradient parity on sampled tokens (each row of Y and dX depends on its own token only)."""
+    (Wg, wsg), (W1, W3, W2), sh = _weights(wl.seed, wl.E, wl.I, wl.d, wl.I_s, wl.bf16)
+    K = wl.K
+    cand = np.sort(np.random.default_rng(7).choice(wl.N, min(wl.N, 2 * n_sample), replace=False))
+    L64 = O.gate_logits(X[cand], Wg)
+    assert_close_abs(L[cand], L64, 1e-4, "L")
+    # backward parity needs the fp64 logits to pick the same experts as the device's fp32 logits
+    same = np.all(O.c2r_route(L64, sets, K)[0] == idx[cand], axis=1)
+    assert same.mean() > 0.9
+    S = cand[same][:n_sample]
+    n = S.size
+    f = O.layer_fwd(X[S], Wg, W1, W3, W2, sets, K, expert_rank=rank, row_align=1, shared=sh, wsg=wsg)
+    assert np.array_equal(f["idx"], idx[S])
+    rows_dev = lay.host("row_of_slot").reshape(wl.N, K)[S].reshape(-1)
+    rows_ref = f["row_of_slot"].reshape(-1)
+    assert_close_elem(_dev_rows(lay.t["H"], rows_dev), f["H"][rows_ref], what="H")
+    assert_close_rms(_dev_rows(lay.t["Yp"], rows_dev), f["Yp"][rows_ref], 5e-2, "Yp", out_bf16=False)
+    assert np.array_equal(_dev_rows(lay.t["Xp"], rows_dev), X[S].astype(np.float64).repeat(K, axis=0))
+    assert_close_rms(_dev_rows(lay.t["Y"], S), f["Y"], 2e-2, "Y")
+    g = O.layer_bwd(X[S], Wg, W1, W3, W2, f, dY[S], shared=sh, wsg=wsg)
+    assert_close_rms(_dev_rows(lay.t["dw"], S), g["dw"], 2e-2, "dw", out_bf16=False)
+    dl_ref = np.take_along_axis(g["dL"], f["idx"], axis=1)
+    assert_close_rms(_dev_rows(lay.t["dl"], S), dl_ref, 2e-2, "dl", out_bf16=False)
+    assert_close_elem(_dev_rows(lay.t["dYp"], rows_dev), g["dYp"][rows_ref], what="dYp")
+    assert_close_rms(_dev_rows(lay.t["dXp"], rows_dev), g["dXp"][rows_ref], 5e-2, "dXp", out_bf16=False)
+    assert_close_rms(_dev_rows(lay.t["dX"], S), g["dX"], 2e-2, "dX")
+    if wl.I_s:
+        assert_close_abs(_dev_rows(lay.t["z"], S), f["z"], 1e-4, "z")
+        assert_close_rms(_dev_rows(lay.t["dz"], S), g["dz"], 2e-2, "dz", out_bf16=False)
+        assert_close_rms(_dev_rows(lay.t["Ys"], S), f["Ys"], 5e-2, "Ys", out_bf16=False)
+
+
+def _check_expert_grads(wl, lay, X, dY, w_ref, counts, offsets, sor, experts):
+    """All three weight gradients of whole experts: the contraction runs over every row routed to them."""
+    _, (W1, W3, W2), _ = _weights(wl.seed, wl.E, wl.I, wl.d, wl.I_s, wl.bf16)
+    K = wl.K
+    dW1_dev, dW3_dev = lay.unpacked_grads()[:2]
+    for e in experts:
+        r0, n = int(offsets[e]), int(counts[e])
+        slots = sor[r0:r0 + n]
+        tok, k = slots // K, slots % K
+        Xe = X[tok].astype(np.float64)
+        dYpe = w_ref[tok, k][:, None] * dY[tok].astype(np.float64)
+        cnt, off = np.array([n]), np.array([0, n])
+        A, B, H, _ = O.swiglu_fwd(Xe, cnt, off, W1[e:e + 1], W3[e:e + 1], W2[e:e + 1])
+        dXp, dW1, dW3, dW2 = O.swiglu_bwd(Xe, cnt, off, W1[e:e + 1], W3[e:e + 1], W2[e:e + 1], A, B, dYpe)
+        assert_close_elem(lay.t["H"][r0:r0 + n].float().cpu().numpy(), H, what=f"H[{e}]")
+        assert_close_rms(lay.t["dXp"][r0:r0 + n].cpu().numpy(), dXp, 5e-2, f"dXp[{e}]", out_bf16=False)
+        # error scale of each gradient element: sqrt(sum over the expert's rows of (term)^2), see assert_close_contraction
+        sg = O.sigmoid(A)
+        dH = dYpe @ np.asarray(W2[e], np.float64)
+        dA, dB = dH * B * (sg * (1.0 + A * (1.0 - sg))), dH * (A * sg)
+        X2 = Xe ** 2
+        assert_close_contraction(lay.t["dW2"][e].float().cpu().numpy(), dW2[0], np.sqrt((dYpe ** 2).T @ (H ** 2)), f"dW2[{e}]")
+        assert_close_contraction(dW1_dev[e].float().cpu().numpy(), dW1[0], np.sqrt((dA ** 2).T @ X2), f"dW1[{e}]")
+        assert_close_contraction(dW3_dev[e].float().cpu().numpy(), dW3[0], np.sqrt((dB ** 2).T @ X2), f"dW3[{e}]")
+        # the rest of the expert's 128-row segment is padding and stays zero
+        pad_end = r0 + -(-n // lay.cfg.row_align) * lay.cfg.row_align
+        assert not lay.t["Xp"][r0 + n:pad_end].any() and not lay.t["dYp"][r0 + n:pad_end].any()
+
+
+def _check_shared_slabs(wl, lay, X, dY, slabs, width=64):
+    """Column slabs of the shared expert's weight gradients: channels [j0, j0+width) of a SwiGLU
+    MLP form an independent sub-expert, which the oracle evaluates over all N tokens."""
+    (Wg, wsg), _, (Ws1, Ws3, Ws2) = _weights(wl.seed, wl.E, wl.I, wl.d, wl.I_s, wl.bf16)
+    X64 = X.astype(np.float64)
+    z = X64 @ wsg.astype(np.float64)
+    dYs = O.sigmoid(z)[:, None] * dY.astype(np.float64)
+    d1_dev, d3_dev = lay.unpacked_grads()[2:]
+    for j0 in slabs:
+        sl = slice(j0, j0 + width)
+        A, B, H, _ = O.dense_swiglu(X64, Ws1[sl], Ws3[sl], Ws2[:, sl])
+        _, dW1, dW3, dW2 = O.dense_swiglu_bwd(X64, Ws1[sl], Ws3[sl], Ws2[:, sl], A, B, dYs)
+        assert_close_elem(lay.t["Hs"][:, sl].float().cpu().numpy(), H, what=f"Hs[:, {j0}:]")
+        assert_close_rms(d1_dev[sl].float().cpu().numpy(), dW1, 2e-2, f"dWs1[{j0}:]")
+        assert_close_rms(d3_dev[sl].float().cpu().numpy(), dW3, 2e-2, f"dWs3[{j0}:]")
+        assert_close_rms(lay.t["dWs2"][0][:, sl].float().cpu().numpy(), dW2, 2e-2, f"dWs2[:, {j0}:]")
+
+
+@pytest.mark.parametrize("name", ["c3", "c2", "c5"])
+def test_fullsize_train_step(name):
+    wl = G.WORKLOADS[name]
+    lay, cal, X, dY = _run(wl)
+    sets, part, rank = _check_calibration(wl, cal)
+    L, idx, w_ref, counts, offsets, ros, sor = _check_integer_path(wl, lay, sets, part, rank)
+    assert int(counts.sum()) == wl.N * wl.K
+    _check_sampled_tokens(wl, lay, X, dY, L, idx, sets, rank, n_sample=64)
+    order = np.argsort(counts)
+    _check_expert_grads(wl, lay, X, dY, w_ref, counts, offsets, sor, experts=[int(order[0]), int(order[-1])])
+    if wl.I_s:
+        _check_shared_slabs(wl, lay, X, dY, slabs=[128, wl.I_s - 64] if wl.N <= 16384 else [wl.I_s - 64])
+    # any-size properties: the softmax backward gives sum_k dl[t,k] = 0, hence sum_e dWg[e,:] = 0
+    dWg = lay.host("dWg").astype(np.float64)
+    assert np.abs(dWg.sum(axis=0)).max() <= 1e-3 * np.abs(dWg).max()
+    for name_ in ("Y", "dX", "dW2", "dW13p"):
+        assert torch.isfinite(lay.t[name_].float()).all(), name_

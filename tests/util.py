@@ -36,6 +36,25 @@ def assert_close_rms(got, ref, frac=2e-2, what="", out_bf16=True, rms_frac=5e-3)
     assert erms <= rms_frac * rms, f"{what}: RMS(err)={erms:.3e} > {rms_frac}*RMS(ref)={rms_frac * rms:.3e}"
 
 
+def assert_close_contraction(got, ref, Q, what="", frac=2e-2, sigmas=6.0, rms_frac=5e-3):
+    """bf16 bar for a result that contracts n bf16-stored products, ref = sum_r a_r x_r (a weight
+    gradient).  Each stored a_r went through three bf16 roundings (dYp, the saved local derivative,
+    dA), i.e. carries a relative error of standard deviation ~2^-8, so even exact arithmetic between
+    the roundings leaves an error of standard deviation 2^-8 * Q on the sum, Q = sqrt(sum_r (a_r x_r)^2)
+    (about RMS(ref) for a typical element, larger where few large terms dominate).  Every element:
+    |err| <= 2^-8 |ref| + max(frac * RMS(ref), sigmas * 2^-8 * Q); and RMS(err) <= rms_frac * RMS(ref)."""
+    got = np.asarray(got, np.float64); ref = np.asarray(ref, np.float64); Q = np.asarray(Q, np.float64)
+    assert got.shape == ref.shape == Q.shape, (what, got.shape, ref.shape, Q.shape)
+    assert np.isfinite(got).all(), what
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    err = np.abs(got - ref)
+    tol = 2.0 ** -8 * np.abs(ref) + np.maximum(frac * rms, sigmas * 2.0 ** -8 * Q)
+    worst = float(np.max(err - tol))
+    assert worst <= 0.0, f"{what}: max|err|={err.max():.3e} ({err.max() / rms:.4f} RMS), over tolerance by {worst:.3e}"
+    erms = float(np.sqrt(np.mean(err ** 2)))
+    assert erms <= rms_frac * rms, f"{what}: RMS(err)={erms:.3e} > {rms_frac}*RMS(ref)={rms_frac * rms:.3e}"
+
+
 def assert_close_abs(got, ref, tol=1e-4, what=""):
     """fp32 bar: max |err| <= tol."""
     got = np.asarray(got, np.float64); ref = np.asarray(ref, np.float64)
