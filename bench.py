@@ -146,7 +146,9 @@ def build_layer(wl, device, profile=True, keep=False):
 
 
 def breakdown(lay, reps=3):
-    """Per-call device time (ms) of one step, each C-ABI call bracketed by CUDA events."""
+    """Per-call device time (ms) of one step: the calls c2r_train_step chains, issued one by one on
+    the same stream with a CUDA event between them, `reps` steps back to back (a sustained loop,
+    so the GEMM figures see the same power-capped clocks as the timed region)."""
     import torch
     from paper_2504_01337_b200 import binding as B
     c, t = lay.cfg, lay.t
@@ -199,6 +201,66 @@ def breakdown(lay, reps=3):
         for i, (n, _) in enumerate(calls):
             acc[n] += evs[i].elapsed_time(evs[i + 1])
     return {n: v / reps for n, v in acc.items()}
+
+
+def dispatch_report(L, mask, Cm_host, E, K, T, partitions=(2, 4, 8)):
+    """Conventional Top-K and C2R on the same fp32 logits L [n,E] (device): per-expert load imbalance
+    and the rows an all-to-all would carry at several expert-parallel degrees (greedy placement
+    from the calibration matrix), all computed by the library."""
+    import torch
+    from paper_2504_01337_b200 import binding as B
+    n = L.shape[0]
+    dev = L.device
+    i32 = dict(dtype=torch.int32, device=dev)
+    idx, w = torch.empty((n, K), **i32), torch.empty((n, K), dtype=torch.float32, device=dev)
+    counts, offsets = torch.empty(E, **i32), torch.empty(E + 1, **i32)
+    ros = torch.empty(n * K, **i32)
+    out = {}
+    for name, m in (("topk", None), ("c2r", mask)):
+        cfg = B.make_config(n, 8, E, 16, K, T, 1, 0, B.F32, 1)
+        B.route(cfg, L, m, idx, w)
+        sor = torch.empty(B.permuted_rows(cfg), **i32)
+        ws = torch.empty(max(1, B.workspace_bytes(cfg, B.WS_PERMUTE)), dtype=torch.uint8, device=dev)
+        B.permute(cfg, idx, None, None, counts, offsets, ros, sor, None, None, ws)
+        c = counts.cpu().numpy().astype(np.float64)
+        rep = {"load_max_over_mean": float(c.max() / c.mean()), "load_cv": float(c.std() / c.mean()),
+               "empty_experts": int((c == 0).sum())}
+        for P in partitions:
+            cP = B.make_config(n, 8, E, 16, K, T, P, 0, B.F32, 1)
+            part, rank = torch.zeros(E, dtype=torch.int32), torch.zeros(E, dtype=torch.int32)
+            B.place_experts(cP, Cm_host, 0, part, rank)
+            tot = torch.zeros(4, dtype=torch.int64, device=dev)
+            sn = torch.zeros((P, P), dtype=torch.int64, device=dev)
+            sd = torch.zeros((P, P), dtype=torch.int64, device=dev)
+            B.dispatch_volume(cP, idx, part.to(dev), tot, sn, sd)
+            t = [int(v) for v in tot.cpu().tolist()]
+            rep[f"P{P}"] = {"naive": t[0], "dedup": t[1], "naive_cross": t[2], "dedup_cross": t[3],
+                            "redundancy": 1.0 - t[1] / max(t[0], 1)}
+        out[name] = rep
+    out["c2r_dedup_cross_vs_topk"] = {f"P{P}": out["c2r"][f"P{P}"]["dedup_cross"] / max(out["topk"][f"P{P}"]["dedup_cross"], 1)
+                                      for P in partitions}
+    return out
+
+
+def skew_report(wl4, device):
+    """The skewed-routing stress workload (directly drawn logits with a Zipf-like expert bias and a
+    block bonus): profile on its calibration logits, then Top-K vs C2R side by side."""
+    import torch
+    from paper_2504_01337_b200 import binding as B
+    from paper_2504_01337_b200 import inputs as G
+    L = torch.from_numpy(G.skewed_logits(wl4)).to(device)
+    Lc = torch.from_numpy(G.skewed_logits(wl4, calib=True)).to(device)
+    n, E, K, T = Lc.shape[0], wl4.E, wl4.K, wl4.T
+    cfg = B.make_config(n, 8, E, 16, K, T, 1, 0, B.F32, 1)
+    idx = torch.empty((n, K), dtype=torch.int32, device=device)
+    w = torch.empty((n, K), dtype=torch.float32, device=device)
+    Cm = torch.zeros((E, E), dtype=torch.int32, device=device)
+    I_T = torch.zeros((E, T), dtype=torch.int32, device=device)
+    mask = torch.zeros((E,), dtype=torch.int64, device=device)
+    B.route(cfg, Lc, None, idx, w)
+    B.collab_count(cfg, idx, n, Cm)
+    B.collab_sets(cfg, Cm, I_T, mask)
+    return dispatch_report(L, mask, Cm.cpu(), E, K, T)
 
 
 def cpu_oracle_step(wl, n_tok, state=None):
@@ -263,6 +325,12 @@ def run_reference(args, wl):
     }))
 
 
+# DRAM bytes per launch of tc_gemm_kernel (dram__bytes_read.sum + dram__bytes_write.sum averaged over
+# the 12 launches of a step) from the ncu launch list of this very command, summarised under
+# profiles/.  Keyed by workload; None where no capture of the current kernel exists.
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = {"c3": None}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -274,9 +342,11 @@ def main():
     ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
+    ap.add_argument("--no-reports", action="store_true", help="skip the Top-K vs C2R dispatch reports")
     args = ap.parse_args()
 
     from paper_2504_01337_b200 import inputs as G
+    from paper_2504_01337_b200 import replicas as RP
     wl = G.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)
@@ -286,45 +356,39 @@ def main():
     import torch.distributed as dist
     from paper_2504_01337_b200 import binding as B  # raises if libc2r.so is missing
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = RP.env_rank()
     device = f"cuda:{local}"
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(device))
 
-    # every rank owns an independent data-parallel shard: same parameters, its own batch seed
-    import dataclasses
-    wl_rank = dataclasses.replace(wl, seed=wl.seed + 1000 * rank) if rank else wl
-    lay = build_layer(wl, device)
-    X_host = torch.from_numpy(G.hidden(wl_rank)).to(torch.bfloat16 if wl.bf16 else torch.float32).pin_memory()
-    dY_host = torch.from_numpy(G.grad_out(wl_rank)).to(X_host.dtype).pin_memory()
+    # every rank is an independent data-parallel replica: same parameters, its own batch
+    wl_rank = RP.rank_workload(wl, rank)
+    lay, cal = build_layer(wl, device, keep=True)
+    if args.workload == "c5":
+        # large-batch training step: the sets refreshed from this step's routing (Eq. 2, Eq. 4) are the
+        # ones the next step routes with (the refresh is the last thing a step enqueues)
+        mask_cal = cal["mask"].clone()
+        lay.t["mask_next"] = lay.t["mask"]
+        lay._bufs = None
+    hdt = torch.bfloat16 if wl.bf16 else torch.float32
+    X_host = torch.from_numpy(G.hidden(wl_rank)).to(hdt).pin_memory()
+    dY_host = torch.from_numpy(G.grad_out(wl_rank)).to(hdt).pin_memory()
     lay.set_input(X_host.to(device), dY_host.to(device))
     Y_host = torch.empty_like(X_host).pin_memory()
     dX_host = torch.empty_like(X_host).pin_memory()
     torch.cuda.synchronize()
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-
-    def max_over_ranks(ms):
-        if world > 1:
-            tns = torch.tensor([ms], dtype=torch.float64, device=device)
-            dist.all_reduce(tns, op=dist.ReduceOp.MAX)
-            return float(tns.item())
-        return ms
 
     lib_launches = getattr(B.lib, "c2r_launch_count", None)
 
     # ---- device-resident timing ----------------------------------------------------------------
     sampler = ClockSampler(local)
     sampler.start()
-    for _ in range(max(args.warmup, 3)):
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
         lay.train_step()
     torch.cuda.synchronize()
-    barrier()
+    RP.barrier()
     sampler.mark_begin()
     launches0 = int(lib_launches()) if lib_launches else 0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -335,35 +399,62 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     sampler.mark_end()
-    barrier()
+    RP.barrier()
     launches = (int(lib_launches()) - launches0) if lib_launches else None
     clocks = sampler.stop()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
-    ms_step = ms_total / args.steps
-    value = world * wl.N / (ms_step * 1e-3)
+    ms_step = RP.max_over_ranks(e0.elapsed_time(e1), device) / args.steps
+    value = RP.whole_job_rate(wl.N, world, ms_step)
     status = int(lay.t["status"].item())
 
     # ---- end to end: pinned host inputs in, results out, every step ----------------------------
-    e2e_steps = max(3, min(args.steps, 10))
-    Xd, dYd = lay.t["X"], lay.t["dY"]
+    # Two slots of (X, dY, Y, dX) on the device and three streams: while step i computes, the inputs
+    # of step i+1 arrive and the results of step i-1 leave.
+    e2e_steps = max(3, min(args.steps, 20))
+    comp = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    slots = []
+    for k in range(2):
+        tk = dict(lay.t)
+        if k:
+            for name in ("X", "dY", "Y", "dX"):
+                tk[name] = torch.empty_like(lay.t[name])
+        slots.append(dict(t=tk, bufs=B.make_layer_buffers(tk), in_ready=torch.cuda.Event(), done=torch.cuda.Event(),
+                          out_done=torch.cuda.Event()))
+    for sl in slots:
+        sl["done"].record(comp)
+        sl["out_done"].record(comp)
 
-    def e2e_step():
-        Xd.copy_(X_host, non_blocking=True)
-        dYd.copy_(dY_host, non_blocking=True)
-        lay.train_step()
-        Y_host.copy_(lay.t["Y"], non_blocking=True)
-        dX_host.copy_(lay.t["dX"], non_blocking=True)
+    def e2e_step(i):
+        sl = slots[i & 1]
+        t = sl["t"]
+        with torch.cuda.stream(s_in):
+            s_in.wait_event(sl["done"])  # the step that last read this slot's inputs has finished
+            t["X"].copy_(X_host, non_blocking=True)
+            t["dY"].copy_(dY_host, non_blocking=True)
+            sl["in_ready"].record(s_in)
+        comp.wait_event(sl["in_ready"])
+        comp.wait_event(sl["out_done"])  # this slot's previous results have left
+        B.train_step(lay.cfg, sl["bufs"])
+        sl["done"].record(comp)
+        with torch.cuda.stream(s_out):
+            s_out.wait_event(sl["done"])
+            Y_host.copy_(t["Y"], non_blocking=True)
+            dX_host.copy_(t["dX"], non_blocking=True)
+            sl["out_done"].record(s_out)
 
-    e2e_step()
+    for i in range(2):
+        e2e_step(i)
     torch.cuda.synchronize()
-    barrier()
+    RP.barrier()
     e0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    for sl in slots:
+        comp.wait_event(sl["out_done"])
     e1.record()
     torch.cuda.synchronize()
-    barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+    RP.barrier()
+    e2e_ms = RP.max_over_ranks(e0.elapsed_time(e1), device) / e2e_steps
     nbytes = X_host.numel() * X_host.element_size()
 
     out = None
@@ -373,32 +464,47 @@ def main():
         vol = lay.host("volume")
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if wl.bf16 else "f32", "data": "synthetic",
             "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "E": wl.E, "I": wl.I, "K": wl.K, "T": wl.T,
-                       "P": wl.P, "I_s": wl.I_s, "row_align": lay.cfg.row_align, "parallelism": f"dp{world}",
-                       "step": "fwd+bwd+collab refresh", "l2": "working set (>1 GB weights + activations) exceeds the 126 MB L2"},
+                       "P": wl.P, "I_s": wl.I_s, "row_align": lay.cfg.row_align, "parallelism": f"dp{world} (replicas)",
+                       "step": "fwd+bwd+collab refresh (c2r_train_step)",
+                       "l2": "working set (>1 GB weights + activations) exceeds the 126 MB L2"},
             "clocks": clocks,
-            "e2e": {"value": world * wl.N / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 2 * nbytes,
-                    "d2h_bytes_per_step": 2 * nbytes, "ms_per_step": e2e_ms},
+            "e2e": {"value": RP.whole_job_rate(wl.N, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": 2 * nbytes,
+                    "d2h_bytes_per_step": 2 * nbytes, "ms_per_step": e2e_ms,
+                    "how": "c2r_train_step on double-buffered inputs/outputs; H2D of X,dY and D2H of Y,dX every step on side streams"},
             "gpu_launches": launches,
             "status_word": status,
             "step_tflops": fl_step / (ms_step * 1e-3) / 1e12,
             "dispatch": {"naive": int(vol[0]), "dedup": int(vol[1]), "redundancy": 1.0 - vol[1] / max(vol[0], 1)},
         }
         if not args.no_breakdown:
-            bd = breakdown(lay)
+            bd = breakdown(lay, reps=max(3, min(args.steps, 30)))
             out["breakdown_ms"] = {k: round(v, 4) for k, v in bd.items()}
-            gemm_ms = sum(v for k, v in bd.items() if k in ("swiglu_fwd", "swiglu_bwd", "shared_fwd", "shared_bwd"))
+            gemm_calls = [k for k in ("swiglu_fwd", "swiglu_bwd", "shared_fwd", "shared_bwd") if k in bd]
+            gemm_ms = sum(bd[k] for k in gemm_calls)
+            n_launch = 6 * len(gemm_calls) // 2  # 2 forward + 4 backward launches per expert group
             ach = fl_step / (gemm_ms * 1e-3) / 1e12
             peak = peaks["bf16_tflops_sustained"]
             out["roofline"] = {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                               "frac": ach / peak, "traffic": None, "peak_source": peaks["source"] + " sustained",
-                               "kernel": "grouped SwiGLU GEMMs (routed + shared, fwd + bwd)"}
+                               "frac": ach / peak, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH.get(wl.name),
+                               "peak_source": peaks["source"] + " sustained (bf16_tflops_sustained; burst %.0f)" % peaks["bf16_tflops"],
+                               "kernel": "tc_gemm_kernel (grouped SwiGLU GEMMs, routed + shared, fwd + bwd)",
+                               "launches_per_step": n_launch, "avg_launch_ms": gemm_ms / n_launch,
+                               "flops_per_launch": fl_step / n_launch}
             es = 2 if wl.bf16 else 4
-            hb = {"permute": wl.N * wl.d * es * (wl.K + 1), "combine": wl.N * wl.d * es * (wl.K + 1 + (1 if wl.I_s else 0))}
+            sh = 1 if wl.I_s else 0
+            hb = {"permute": wl.N * wl.d * es * (wl.K + 1),
+                  "combine": wl.N * wl.d * (4 * wl.K + 4 * sh + es),
+                  "combine_bwd": wl.N * wl.d * (4 * wl.K + 4 * sh + es + es * wl.K + es * sh),
+                  "unpermute_grad": wl.N * wl.d * (4 * wl.K + 4 * sh + es)}
             out["hbm_gbs"] = {k: hb[k] / (bd[k] * 1e-3) / 1e9 for k in hb}
             out["hbm_frac_of_measured"] = {k: v / peaks["hbm_gbs"] for k, v in out["hbm_gbs"].items()}
+        if not args.no_reports:
+            out["dispatch_report"] = dispatch_report(lay.t["L"], lay.t["mask"] if args.workload != "c5" else mask_cal,
+                                                     cal["C"].cpu(), wl.E, wl.K, wl.T)
+            out["skew_report_c4"] = skew_report(G.WORKLOADS["c4"], device)
         if not args.no_cpu_baseline and world == 1:
             n_tok = args.cpu_baseline_tokens
             dt, _ = cpu_oracle_step(wl, n_tok)

@@ -185,3 +185,82 @@ def test_fullsize_train_step(name):
     assert np.abs(dWg.sum(axis=0)).max() <= 1e-3 * np.abs(dWg).max()
     for name_ in ("Y", "dX", "dW2", "dW13p"):
         assert torch.isfinite(lay.t[name_].float()).all(), name_
+
+
+def test_c4_skewed_routing_topk_vs_c2r_and_forward():
+    """Skewed-routing stress workload (Zipf-like expert bias + block bonus on directly drawn logits):
+    conventional Top-4 and C2R side by side -- routing, load, dispatch volume at P = 2, 4, 8 -- all
+    bit-exact against the oracle; then the forward pass under the C2R routing, where almost every
+    token lands on the same few experts and most experts receive nothing."""
+    from paper_2504_01337_b200 import binding as b
+    from paper_2504_01337_b200.layer import C2RLayer, to_device
+    wl = G.WORKLOADS["c4"]
+    N, E, K, T = wl.N, wl.E, wl.K, wl.T
+    L, Lcal = G.skewed_logits(wl), G.skewed_logits(wl, calib=True)
+    Ld, Lcd = torch.from_numpy(L).cuda(), torch.from_numpy(Lcal).cuda()
+    cfg = b.make_config(N, wl.d, E, wl.I, K, T, wl.P, wl.I_s, b.BF16, 128)
+    i32 = dict(dtype=torch.int32, device="cuda")
+    idx, w = torch.zeros((N, K), **i32), torch.zeros((N, K), device="cuda")
+    Cm, I_T = torch.zeros((E, E), **i32), torch.zeros((E, T), **i32)
+    mask = torch.zeros((E,), dtype=torch.int64, device="cuda")
+    # profiling on the calibration logits under conventional Top-K
+    b.route(cfg, Lcd, None, idx, w)
+    b.collab_count(cfg, idx, N, Cm)
+    b.collab_sets(cfg, Cm, I_T, mask)
+    idxc_ref, _ = O.topk_route(Lcal, K)
+    C_ref = O.collab_count(idxc_ref, E)
+    sets = O.collab_sets(C_ref, T)
+    assert np.array_equal(Cm.cpu().numpy(), C_ref) and np.array_equal(I_T.cpu().numpy(), sets)
+    ws = torch.empty(b.workspace_bytes(cfg, b.WS_PERMUTE), dtype=torch.uint8, device="cuda")
+    counts, offsets = torch.zeros(E, **i32), torch.zeros(E + 1, **i32)
+    ros, sor = torch.zeros(N * K, **i32), torch.zeros(b.permuted_rows(cfg), **i32)
+    status = torch.zeros(1, **i32)
+    report = {}
+    for mode, m in (("topk", None), ("c2r", mask)):
+        b.route(cfg, Ld, m, idx, w, None, status)
+        ridx, rw = (O.topk_route(L, K) if m is None else O.c2r_route(L, sets, K))
+        assert np.array_equal(idx.cpu().numpy(), ridx)
+        assert_close_abs(w.cpu().numpy(), rw, 1e-5, "w " + mode)
+        b.permute(cfg, idx, None, None, counts, offsets, ros, sor, None, status, ws)
+        rc, ro, rros, rsor = O.permute_index(ridx, E, None, 128)
+        assert np.array_equal(counts.cpu().numpy(), rc) and np.array_equal(ros.cpu().numpy(), rros)
+        report[mode] = {"load": O.load_stats(rc)}
+        for P in (2, 4, 8):
+            cP = b.make_config(N, wl.d, E, wl.I, K, T, P, wl.I_s, b.BF16, 128)
+            part, rank = torch.zeros(E, dtype=torch.int32), torch.zeros(E, dtype=torch.int32)
+            b.place_experts(cP, Cm.cpu(), 0, part, rank)
+            part_ref, rank_ref = O.place_experts(C_ref, P)
+            assert np.array_equal(part.numpy(), part_ref) and np.array_equal(rank.numpy(), rank_ref)
+            tot = torch.zeros(4, dtype=torch.int64, device="cuda")
+            sn, sd = torch.zeros((P, P), dtype=torch.int64, device="cuda"), torch.zeros((P, P), dtype=torch.int64, device="cuda")
+            b.dispatch_volume(cP, idx, part.cuda(), tot, sn, sd)
+            v = O.dispatch_volume(ridx, part_ref, P)
+            assert tot.cpu().tolist() == [v["naive"], v["dedup"], v["naive_x"], v["dedup_x"]]
+            assert np.array_equal(sn.cpu().numpy(), v["send_naive"]) and np.array_equal(sd.cpu().numpy(), v["send_dedup"])
+            report[mode][P] = v["dedup"]
+        assert int(status.item()) == 0
+    # the constraint never adds partitions per token on this workload, and the skew is extreme
+    assert all(report["c2r"][P] <= report["topk"][P] for P in (2, 4, 8))
+    assert report["c2r"]["load"]["max_over_mean"] > 10 and int((rc == 0).sum()) > 0
+    # forward under the C2R routing just computed (idx, w still hold it), greedy placement at P = 4
+    (Wg, wsg), (W1, W3, W2), sh = _weights(wl.seed, E, wl.I, wl.d, wl.I_s, wl.bf16)
+    lay = C2RLayer(N, wl.d, E, wl.I, K, T, wl.P, wl.I_s, True, backward=False)
+    lay.set_params(Wg, W1, W3, W2, wsg, sh)
+    X = G.hidden(wl)
+    t = lay.t
+    t["X"] = to_device(X, True)
+    part_ref, rank_ref = O.place_experts(C_ref, wl.P)
+    rank_d = torch.from_numpy(rank_ref.astype(np.int32)).cuda()
+    b.gate_logits(cfg, t["X"], t["Wg"], t["wsg"], t["L"], t["z"])  # only z (the shared-expert gate) is used from this call
+    b.permute(cfg, idx, rank_d, t["X"], t["counts"], t["offsets"], t["row_of_slot"], t["slot_of_row"], t["Xp"], status, ws)
+    b.grouped_swiglu_fwd(cfg, E, wl.I, lay.R, t["Xp"], t["counts"], t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["Yp"], status)
+    b.grouped_swiglu_fwd(cfg, 1, wl.I_s, N, t["X"], t["s_counts"], t["s_offsets"], t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["Ys"], status)
+    b.combine(cfg, t["Yp"], w, t["row_of_slot"], t["Ys"], t["z"], t["Y"])
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    S = np.sort(np.random.default_rng(3).choice(N, 64, replace=False))
+    f = O.layer_fwd(X[S], Wg, W1, W3, W2, sets, K, expert_rank=rank_ref, row_align=1, shared=sh, wsg=wsg, logits=L[S])
+    assert np.array_equal(f["idx"], ridx[S])
+    assert_close_rms(_dev_rows(t["Y"], S), f["Y"], 2e-2, "Y")
+    rows_dev = t["row_of_slot"].cpu().numpy().reshape(N, K)[S].reshape(-1)
+    assert_close_elem(_dev_rows(t["H"], rows_dev), f["H"][f["row_of_slot"].reshape(-1)], what="H")
