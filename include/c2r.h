@@ -104,6 +104,12 @@ int c2r_collab_count(const c2r_config* cfg, const int32_t* idx, int64_t n_tokens
  * (ties: lower j); mask[i] has exactly those bits set.  C [E,E] int32; I_T [E,T] int32; mask [E] uint64. */
 int c2r_collab_sets(const c2r_config* cfg, const int32_t* C, int32_t* I_T, uint64_t* mask, void* stream);
 
+/* Sec. 3.2, Eq. 3 (collaboration degree): degree[i] = - sum_{j != i} p_ij ln p_ij with
+ * p_ij = C[i,j] / sum_{j != i} C[i,j] (the normaliser runs over the same j != i as the sum; natural
+ * logarithm; 0 ln 0 = 0; a row without co-activations gives 0).  Lower = more specialised collaboration.
+ * C [E,E] int32; out: degree [E] float; mean (one float, may be NULL) = the layer's average over experts. */
+int c2r_collab_degree(const c2r_config* cfg, const int32_t* C, float* degree, float* mean, void* stream);
+
 /* Sec. 3.4 (co-locate closely collaborating experts on one device).  HOST function, host arrays.
  * mode 0 (greedy): partition p holds floor(E/P) + (p < E mod P) experts; it is seeded with the
  * unassigned expert of largest C[e,e] and grown by the unassigned expert with the largest summed

@@ -53,7 +53,7 @@ class LayerBuffers(C.Structure):
 
 EXPORTS = [
     "c2r_workspace_bytes", "c2r_permuted_rows", "c2r_last_cuda_error", "c2r_launch_count", "c2r_gate_logits", "c2r_route",
-    "c2r_collab_count", "c2r_collab_sets", "c2r_place_experts", "c2r_permute", "c2r_pack_weights",
+    "c2r_collab_count", "c2r_collab_sets", "c2r_collab_degree", "c2r_place_experts", "c2r_permute", "c2r_pack_weights",
     "c2r_unpack_weights", "c2r_grouped_swiglu_fwd", "c2r_grouped_swiglu_bwd", "c2r_combine", "c2r_combine_bwd",
     "c2r_route_bwd", "c2r_gate_bwd", "c2r_unpermute_grad", "c2r_dispatch_volume", "c2r_layer_fwd",
     "c2r_layer_bwd", "c2r_train_step", "c2r_permute_static",
@@ -72,6 +72,7 @@ _SIGS = {
     "c2r_route": [_CFG] + [_P] * 7,
     "c2r_collab_count": [_CFG, _P, C.c_int64, _P, C.c_int, _P],
     "c2r_collab_sets": [_CFG] + [_P] * 4,
+    "c2r_collab_degree": [_CFG] + [_P] * 4,
     "c2r_place_experts": [_CFG, _P, C.c_int, _P, _P],
     "c2r_permute": [_CFG] + [_P] * 10 + [C.c_size_t, _P],
     "c2r_permute_static": [_CFG] + [_P] * 10,
@@ -147,6 +148,10 @@ def route(cfg, L, mask, idx, w, p=None, status=None):
 
 def collab_count(cfg, idx, n_tokens, Cmat, accumulate=False):
     _call("c2r_collab_count", C.byref(cfg), _ptr(idx), int(n_tokens), _ptr(Cmat), int(accumulate), _stream())
+
+
+def collab_degree(cfg, Cmat, degree, mean=None):
+    _call("c2r_collab_degree", C.byref(cfg), _ptr(Cmat), _ptr(degree), _ptr(mean), _stream())
 
 
 def collab_sets(cfg, Cmat, I_T, mask):

@@ -213,6 +213,37 @@ __global__ void collab_sets_kernel(const int32_t* __restrict__ C, int32_t* __res
   if (lane == 0) mask[i] = m;
 }
 
+// Collaboration degree (Eq. 3): P_i = - sum_{j != i} p_ij ln p_ij with p_ij = c_ij / sum_{j != i} c_ij
+// (a row without co-activations gives 0; 0 ln 0 = 0).  One block; a warp per row, lanes over the
+// columns, and a fixed-order sum over rows for the layer mean.
+__global__ void __launch_bounds__(1024) collab_degree_kernel(const int32_t* __restrict__ C, float* __restrict__ degree,
+                                                             float* __restrict__ mean, int E) {
+  __shared__ float s_deg[64];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int i = warp; i < E; i += 32) {
+    float c0 = (lane < E && lane != i) ? (float)max(C[i * E + lane], 0) : 0.f;
+    float c1 = (lane + 32 < E && lane + 32 != i) ? (float)max(C[i * E + lane + 32], 0) : 0.f;
+    float tot = c0 + c1;
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, off);
+    float h = 0.f;
+    if (tot > 0.f) {
+      const float p0 = c0 / tot, p1 = c1 / tot;
+      if (p0 > 0.f) h -= p0 * logf(p0);
+      if (p1 > 0.f) h -= p1 * logf(p1);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) h += __shfl_xor_sync(0xffffffffu, h, off);
+    if (lane == 0) { s_deg[i] = h; degree[i] = h; }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && mean != nullptr) {
+    float m = 0.f;
+    for (int i = 0; i < E; ++i) m += s_deg[i];
+    *mean = m / (float)E;
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Dispatch volume (Sec. 3.4 / 4.1): distinct (token, partition) pairs vs (token, expert) pairs.
 // ---------------------------------------------------------------------------------------------
@@ -339,6 +370,15 @@ extern "C" int c2r_collab_sets(const c2r_config* cfg, const int32_t* C, int32_t*
   C2R_REQUIRE(cfg->T >= 0 && cfg->T <= cfg->E - 1, C2R_ERR_INVALID_ARG);
   const int warps = 4;
   collab_sets_kernel<<<(cfg->E + warps - 1) / warps, warps * 32, 0, as_stream(stream)>>>(C, I_T, mask, cfg->E, cfg->T);
+  C2R_LAUNCH_CHECK();
+  return C2R_OK;
+}
+
+extern "C" int c2r_collab_degree(const c2r_config* cfg, const int32_t* C, float* degree, float* mean, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(C && degree, C2R_ERR_INVALID_ARG);
+  collab_degree_kernel<<<1, 1024, 0, as_stream(stream)>>>(C, degree, mean, cfg->E);
   C2R_LAUNCH_CHECK();
   return C2R_OK;
 }

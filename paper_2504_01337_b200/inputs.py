@@ -183,3 +183,12 @@ def skewed_logits(wl: Workload, calib: bool = False, n: int | None = None, block
 
 def random_logits(seed: int, n: int, E: int, std: float = 1.0, stream: int = S_MISC) -> np.ndarray:
     return normal(seed, stream, (n, E), std)
+
+
+def random_collab_matrix(seed: int, E: int, high: int = 1 << 20) -> np.ndarray:
+    """A symmetric int32 [E,E] matrix of independent uniform draws: fed to the Top-T selection of
+    Eq. 4 in place of measured co-activation counts it yields uniformly random collaborator sets
+    (the 'random initialisation' control of Sec. 4.1)."""
+    a = integers(seed, S_MISC, (E, E), high).astype(np.int64)
+    a = np.triu(a, 1)
+    return (a + a.T).astype(np.int32)

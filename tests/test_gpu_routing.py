@@ -205,3 +205,38 @@ def test_argument_errors_are_codes_not_faults():
     with pytest.raises(b.C2RError) as e:
         b.permute(cfg, idx, None, None, idx, idx, idx, idx, None, None, None)
     assert e.value.code == -3
+
+
+@pytest.mark.parametrize("E,K,N", [(8, 2, 4096), (60, 4, 16384), (64, 8, 500), (33, 3, 7)])
+def test_collab_degree(E, K, N):
+    """Eq. 3 on the device against the oracle, on measured counts and on degenerate rows."""
+    b = B()
+    idx, _ = O.topk_route(G.random_logits(E + N, N, E), K)
+    Cm = O.collab_count(idx, E).astype(np.int32)
+    Cm[E - 1, :] = 0            # an expert that never fired: degree 0
+    Cm[0, :] = 0; Cm[0, 0] = 9; Cm[0, 1] = 5  # a single collaborator: degree 0
+    cfg = b.make_config(1, 8, E, 16, K, K - 1, 1, 0, b.F32, 1)
+    deg = torch.full((E,), 7.0, device="cuda"); mean = torch.full((1,), 7.0, device="cuda")
+    b.collab_degree(cfg, dev(Cm), deg, mean)
+    ref, ref_mean = O.collab_degree(Cm)
+    assert_close_abs(host(deg), ref, 1e-4, "degree")
+    assert abs(float(mean.item()) - ref_mean) <= 1e-4
+    assert host(deg)[0] == 0.0 and host(deg)[E - 1] == 0.0
+
+
+def test_random_sets_control():
+    """Random-C2R control: Eq. 4 applied to a random matrix gives valid sets (T distinct j != i)
+    that the router accepts, identical on both sides."""
+    b = B()
+    E, T, K, N = 60, 16, 4, 2000
+    Cr = G.random_collab_matrix(4, E)
+    cfg = b.make_config(N, 8, E, 16, K, T, 1, 0, b.F32, 1)
+    I_T = torch.zeros((E, T), dtype=torch.int32, device="cuda")
+    mask = torch.zeros((E,), dtype=torch.int64, device="cuda")
+    b.collab_sets(cfg, dev(Cr), I_T, mask)
+    ref = O.collab_sets(Cr, T)
+    assert np.array_equal(host(I_T), ref)
+    assert all(len(set(r)) == T and i not in r for i, r in enumerate(ref.tolist()))
+    L = G.random_logits(9, N, E)
+    idx, w, _, st = _route_gpu(L, host(mask).view(np.uint64), K, T)
+    assert np.array_equal(idx, O.c2r_route(L, ref, K)[0]) and st == 0
