@@ -261,6 +261,50 @@ def dispatch_volume(idx, part, P):
     }
 
 
+def dedup_dispatch_index(idx, part, P):
+    """Zero-redundancy dispatch of Sec. 3.4: a token is sent ONCE to every partition that hosts at
+    least one of its selected experts and replicated there.  Receive buffer of partition q = the
+    tokens that need it, in token order (hence grouped by source shard); segments laid out in
+    partition order.  Returns recv_counts [P], recv_offsets [P+1], recv_row_of_slot [N*K] (the
+    receive row holding the copy that slot (t,k) reads) and token_of_recv_row [sum recv_counts]."""
+    idx = np.asarray(idx, dtype=np.int64)
+    part = np.asarray(part, dtype=np.int64)
+    N, K = idx.shape
+    members = [[] for _ in range(P)]          # tokens received by each partition, in token order
+    for t in range(N):
+        seen = set()
+        for k in range(K):
+            q = int(part[idx[t, k]])
+            if q not in seen:
+                seen.add(q)
+                members[q].append(t)
+    recv_counts = np.array([len(m) for m in members], dtype=np.int64)
+    recv_offsets = np.zeros(P + 1, dtype=np.int64)
+    recv_offsets[1:] = np.cumsum(recv_counts)
+    token_of_recv_row = np.array([t for m in members for t in m], dtype=np.int64)
+    row_of = {}
+    for q in range(P):
+        for j, t in enumerate(members[q]):
+            row_of[(t, q)] = int(recv_offsets[q]) + j
+    recv_row_of_slot = np.empty(N * K, dtype=np.int64)
+    for t in range(N):
+        for k in range(K):
+            recv_row_of_slot[t * K + k] = row_of[(t, int(part[idx[t, k]]))]
+    return recv_counts, recv_offsets, recv_row_of_slot, token_of_recv_row
+
+
+def dedup_dispatch(X, slot_of_row, recv_row_of_slot, token_of_recv_row):
+    """Stage 1: Xr[j] = X[token_of_recv_row[j]] (what crosses the interconnect, one row per
+    (token, partition)).  Stage 2, local to a partition: Xp[r] = Xr[recv_row_of_slot[slot_of_row[r]]],
+    padding rows zero.  Returns (Xr, Xp)."""
+    X = np.asarray(X)
+    Xr = X[np.asarray(token_of_recv_row, dtype=np.int64)]
+    Xp = np.zeros((slot_of_row.size, X.shape[1]), dtype=X.dtype)
+    live = slot_of_row >= 0
+    Xp[live] = Xr[np.asarray(recv_row_of_slot)[slot_of_row[live]]]
+    return Xr, Xp
+
+
 def load_stats(counts):
     """Load imbalance of per-expert token counts: max/mean and coefficient of variation."""
     c = np.asarray(counts, F64)
