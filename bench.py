@@ -242,6 +242,45 @@ def dispatch_report(L, mask, Cm_host, E, K, T, partitions=(2, 4, 8)):
     return out
 
 
+def dedup_dispatch_timing(lay, reps=5):
+    """The zero-redundancy two-stage dispatch (Sec. 3.4) on the bench batch, timed beside the plain
+    dispatch it replaces: stage 1 writes one row per (token, partition) -- the rows an all-to-all
+    would carry -- and stage 2 replicates inside the partition."""
+    import torch
+    from paper_2504_01337_b200 import binding as B
+    c, t = lay.cfg, lay.t
+    dev = t["X"].device
+    i32 = dict(dtype=torch.int32, device=dev)
+    cap = c.N * min(c.K, c.P)
+    rc, ro = torch.zeros(c.P, **i32), torch.zeros(c.P + 1, **i32)
+    rrs, tok = torch.zeros(c.N * c.K, **i32), torch.zeros(cap, **i32)
+    Xr = torch.empty((cap, c.d), dtype=t["X"].dtype, device=dev)
+    ws = torch.empty(B.workspace_bytes(c, B.WS_DISPATCH_DEDUP), dtype=torch.uint8, device=dev)
+
+    def run_dedup():
+        B.dispatch_dedup(c, t["idx"], t["part"], t.get("expert_rank"), t["X"], t["counts"], t["offsets"], t["row_of_slot"],
+                         t["slot_of_row"], rc, ro, rrs, tok, Xr, t["Xp"], t["status"], ws)
+
+    def run_plain():
+        B.permute(c, t["idx"], t.get("expert_rank"), t["X"], t["counts"], t["offsets"], t["row_of_slot"], t["slot_of_row"],
+                  t["Xp"], t["status"], t["ws"])
+
+    res = {}
+    for name, fn in (("dedup_two_stage", run_dedup), ("plain", run_plain)):
+        fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        res[name + "_ms"] = e0.elapsed_time(e1) / reps
+    res["stage1_rows"] = int(ro[c.P].item())
+    res["plain_rows"] = c.N * c.K
+    res["P"] = c.P
+    return res
+
+
 def skew_report(wl4, device):
     """The skewed-routing stress workload (directly drawn logits with a Zipf-like expert bias and a
     block bonus): profile on its calibration logits, then Top-K vs C2R side by side."""
@@ -505,6 +544,7 @@ def main():
             out["dispatch_report"] = dispatch_report(lay.t["L"], lay.t["mask"] if args.workload != "c5" else mask_cal,
                                                      cal["C"].cpu(), wl.E, wl.K, wl.T)
             out["skew_report_c4"] = skew_report(G.WORKLOADS["c4"], device)
+            out["dedup_dispatch"] = dedup_dispatch_timing(lay)
         if not args.no_cpu_baseline and world == 1:
             n_tok = args.cpu_baseline_tokens
             dt, _ = cpu_oracle_step(wl, n_tok)

@@ -64,7 +64,7 @@ typedef struct c2r_config {
   int32_t flags;     /* reserved, 0 */
 } c2r_config;
 
-enum { C2R_WS_PERMUTE = 0, C2R_WS_GATE_BWD = 1, C2R_WS_LAYER = 2 };
+enum { C2R_WS_PERMUTE = 0, C2R_WS_GATE_BWD = 1, C2R_WS_LAYER = 2, C2R_WS_DISPATCH_DEDUP = 3 };
 
 /* Bytes of scratch the named call needs for this configuration (host function). */
 size_t c2r_workspace_bytes(const c2r_config* cfg, int which);
@@ -129,6 +129,25 @@ int c2r_place_experts(const c2r_config* cfg, const int32_t* C_host, int mode, in
 int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
                 int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp,
                 int32_t* status, void* ws, size_t ws_bytes, void* stream);
+
+/* Sec. 3.4 (zero-redundancy all-to-all), carried out on one device in its two stages.
+ * Stage 1: every token is copied ONCE to each partition that hosts at least one of its selected
+ * experts.  Partition q receives recv_counts[q] rows, in token order, at rows
+ * [recv_offsets[q], recv_offsets[q+1]) of Xr; recv_offsets[P] is the number of rows an all-to-all
+ * would carry (the `dedup` total of c2r_dispatch_volume, against N*K for the plain dispatch).
+ * Stage 2, local to a partition: the per-expert layout of c2r_permute is filled from the receive
+ * buffer, Xp[r,:] = Xr[recv_row_of_slot[slot_of_row[r]],:].  With a partition-major expert_rank a
+ * partition's rows of Xp read only that partition's segment of Xr.
+ * part [E] int32 (expert -> partition, cfg->P partitions); the other inputs as c2r_permute.
+ * out: counts, offsets, row_of_slot, slot_of_row, Xp exactly as c2r_permute writes them (bit-exact);
+ *      recv_counts [P], recv_offsets [P+1] int32; recv_row_of_slot [N*K] int32; token_of_recv_row
+ *      [N*min(K,P)] int32 (-1 beyond recv_offsets[P]); Xr [N*min(K,P), d] T.
+ * X == NULL builds the indices only.  Atomic-free and deterministic.  ws: C2R_WS_DISPATCH_DEDUP bytes. */
+int c2r_dispatch_dedup(const c2r_config* cfg, const int32_t* idx, const int32_t* part, const int32_t* expert_rank,
+                       const void* X, int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row,
+                       int32_t* recv_counts, int32_t* recv_offsets, int32_t* recv_row_of_slot,
+                       int32_t* token_of_recv_row, void* Xr, void* Xp, int32_t* status, void* ws, size_t ws_bytes,
+                       void* stream);
 
 /* c2r_permute without a workspace argument (an addition of this library; the paper has no
  * counterpart).  Same inputs, same outputs and the same bit-exact results as c2r_permute; the

@@ -20,7 +20,7 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 F32, BF16 = 0, 1
-WS_PERMUTE, WS_GATE_BWD, WS_LAYER = 0, 1, 2
+WS_PERMUTE, WS_GATE_BWD, WS_LAYER, WS_DISPATCH_DEDUP = 0, 1, 2, 3
 ERRORS = {-1: "C2R_ERR_INVALID_ARG", -2: "C2R_ERR_UNSUPPORTED_SHAPE", -3: "C2R_ERR_WORKSPACE", -4: "C2R_ERR_CUDA",
           -5: "C2R_ERR_STATIC_SCRATCH"}
 
@@ -56,7 +56,7 @@ EXPORTS = [
     "c2r_collab_count", "c2r_collab_sets", "c2r_collab_degree", "c2r_place_experts", "c2r_permute", "c2r_pack_weights",
     "c2r_unpack_weights", "c2r_grouped_swiglu_fwd", "c2r_grouped_swiglu_bwd", "c2r_combine", "c2r_combine_bwd",
     "c2r_route_bwd", "c2r_gate_bwd", "c2r_unpermute_grad", "c2r_dispatch_volume", "c2r_layer_fwd",
-    "c2r_layer_bwd", "c2r_train_step", "c2r_permute_static",
+    "c2r_layer_bwd", "c2r_train_step", "c2r_permute_static", "c2r_dispatch_dedup",
 ]
 
 _P = C.c_void_p
@@ -76,6 +76,7 @@ _SIGS = {
     "c2r_place_experts": [_CFG, _P, C.c_int, _P, _P],
     "c2r_permute": [_CFG] + [_P] * 10 + [C.c_size_t, _P],
     "c2r_permute_static": [_CFG] + [_P] * 10,
+    "c2r_dispatch_dedup": [_CFG] + [_P] * 16 + [C.c_size_t, _P],
     "c2r_pack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
     "c2r_unpack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
     "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 10,
@@ -172,6 +173,14 @@ def permute_static(cfg, idx, expert_rank, X, counts, offsets, row_of_slot, slot_
     """c2r_permute with the scratch inside the library (no workspace, no allocation anywhere)."""
     _call("c2r_permute_static", C.byref(cfg), _ptr(idx), _ptr(expert_rank), _ptr(X), _ptr(counts), _ptr(offsets),
           _ptr(row_of_slot), _ptr(slot_of_row), _ptr(Xp), _ptr(status), _stream())
+
+
+def dispatch_dedup(cfg, idx, part, expert_rank, X, counts, offsets, row_of_slot, slot_of_row, recv_counts, recv_offsets,
+                   recv_row_of_slot, token_of_recv_row, Xr, Xp, status, ws):
+    _call("c2r_dispatch_dedup", C.byref(cfg), _ptr(idx), _ptr(part), _ptr(expert_rank), _ptr(X), _ptr(counts),
+          _ptr(offsets), _ptr(row_of_slot), _ptr(slot_of_row), _ptr(recv_counts), _ptr(recv_offsets),
+          _ptr(recv_row_of_slot), _ptr(token_of_recv_row), _ptr(Xr), _ptr(Xp), _ptr(status), _ptr(ws),
+          0 if ws is None else ws.numel() * ws.element_size(), _stream())
 
 
 def pack_weights(cfg, n_experts, I, W1, W3, W13p):

@@ -20,6 +20,7 @@ extern "C" size_t c2r_workspace_bytes(const c2r_config* cfg, int which) {
     case C2R_WS_PERMUTE: return align256(permute_ws_bytes(cfg));
     case C2R_WS_GATE_BWD: return align256(gate_bwd_ws_bytes(cfg));
     case C2R_WS_LAYER: return align256(permute_ws_bytes(cfg)) + align256(gate_bwd_ws_bytes(cfg));
+    case C2R_WS_DISPATCH_DEDUP: return align256(dispatch_dedup_ws_bytes(cfg));
     default: return 0;
   }
 }

@@ -59,5 +59,6 @@ int gate_logits_impl(const c2r_config* cfg, const void* X, const void* Wg, const
 
 size_t permute_ws_bytes(const c2r_config* cfg);
 size_t gate_bwd_ws_bytes(const c2r_config* cfg);
+size_t dispatch_dedup_ws_bytes(const c2r_config* cfg);
 
 }  // namespace c2r

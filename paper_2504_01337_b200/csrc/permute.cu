@@ -17,8 +17,9 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
 // Per-warp, per-expert counts of this block's slots.  A warp owns PERM_ITERS*32 consecutive
 // slots; inside a 32-slot group, lanes with equal expert form a peer set (match.any) whose
 // lowest lane adds the set size -- no atomics, and the order of slots is preserved.
+// skip_negative: a key of -1 marks a slot that takes no part (used by the de-duplicated dispatch).
 __device__ __forceinline__ void warp_count(const int32_t* __restrict__ idx, long long NK, int E, int (*warp_cnt)[64],
-                                           int e_reg[PERM_ITERS], int& flags) {
+                                           int e_reg[PERM_ITERS], int& flags, int skip_negative) {
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const long long base = (long long)blockIdx.x * PERM_BLOCK_SLOTS + (long long)w * PERM_ITERS * 32;
 #pragma unroll
@@ -27,7 +28,7 @@ __device__ __forceinline__ void warp_count(const int32_t* __restrict__ idx, long
     int e = -1;
     if (s < NK) {
       e = idx[s];
-      if (e < 0 || e >= E) { flags |= C2R_STATUS_BAD_INDEX; e = min(max(e, 0), E - 1); }
+      if ((e < 0 || e >= E) && !(skip_negative && e == -1)) { flags |= C2R_STATUS_BAD_INDEX; e = min(max(e, 0), E - 1); }
     }
     e_reg[it] = e;
     const uint32_t peers = __match_any_sync(0xffffffffu, e);
@@ -38,13 +39,13 @@ __device__ __forceinline__ void warp_count(const int32_t* __restrict__ idx, long
 
 __global__ void __launch_bounds__(PERM_WARPS * 32) perm_hist_kernel(const int32_t* __restrict__ idx, long long NK, int E,
                                                                     int32_t* __restrict__ block_counts,
-                                                                    int32_t* __restrict__ status) {
+                                                                    int32_t* __restrict__ status, int skip_negative) {
   __shared__ int warp_cnt[PERM_WARPS][64];
   for (int i = threadIdx.x; i < PERM_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
   __syncthreads();
   int e_reg[PERM_ITERS];
   int flags = 0;
-  warp_count(idx, NK, E, warp_cnt, e_reg, flags);
+  warp_count(idx, NK, E, warp_cnt, e_reg, flags, skip_negative);
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
     int s = 0;
@@ -103,13 +104,13 @@ __global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_kernel(const int32_
                                                                     const int32_t* __restrict__ block_base,
                                                                     const int32_t* __restrict__ offsets,
                                                                     int32_t* __restrict__ row_of_slot,
-                                                                    int32_t* __restrict__ slot_of_row) {
+                                                                    int32_t* __restrict__ slot_of_row, int skip_negative) {
   __shared__ int warp_cnt[PERM_WARPS][64];
   for (int i = threadIdx.x; i < PERM_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
   __syncthreads();
   int e_reg[PERM_ITERS];
   int flags = 0;
-  warp_count(idx, NK, E, warp_cnt, e_reg, flags);
+  warp_count(idx, NK, E, warp_cnt, e_reg, flags, skip_negative);
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
     int run = offsets[e] + block_base[(size_t)blockIdx.x * E + e];
@@ -461,13 +462,13 @@ int permute_impl(const c2r_config* cfg, const int32_t* idx, const int32_t* exper
   int32_t* block_counts = (int32_t*)ws;
   C2R_CUDA(cudaMemsetAsync(slot_of_row, 0xFF, sizeof(int32_t) * R, s));
   if (nb > 0) {
-    perm_hist_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, status);
+    perm_hist_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, status, 0);
     C2R_LAUNCH_CHECK();
   }
   perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, cfg->E, expert_rank, cfg->row_align, counts, offsets);
   C2R_LAUNCH_CHECK();
   if (nb > 0) {
-    perm_rank_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, offsets, row_of_slot, slot_of_row);
+    perm_rank_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, offsets, row_of_slot, slot_of_row, 0);
     C2R_LAUNCH_CHECK();
   }
   if (X != nullptr) {
@@ -660,4 +661,177 @@ extern "C" int c2r_permute_static(const c2r_config* cfg, const int32_t* idx, con
                                        slot_of_row, (__nv_bfloat16*)Xp, status, scratch, as_stream(stream));
   return permute_impl<float>(cfg, idx, expert_rank, (const float*)X, counts, offsets, row_of_slot, slot_of_row,
                              (float*)Xp, status, scratch, as_stream(stream));
+}
+
+// ---------------------------------------------------------------------------------------------
+// Zero-redundancy dispatch (Sec. 3.4) in two stages: one copy of a token per partition that hosts
+// any of its experts (what an all-to-all would carry), then replication inside the partition into
+// the per-expert layout.
+// ---------------------------------------------------------------------------------------------
+namespace c2r {
+
+// key[t,k] = partition of slot (t,k) if no earlier slot of the token maps to that partition, else -1.
+__global__ void __launch_bounds__(256) dedup_keys_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ part,
+                                                         int32_t* __restrict__ key, int N, int E, int K, int P) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= N) return;
+  int q[8];
+  for (int k = 0; k < K; ++k) {
+    const int e = min(max(idx[(size_t)t * K + k], 0), E - 1);
+    q[k] = min(max(part[e], 0), P - 1);
+    bool first = true;
+    for (int j = 0; j < k; ++j) first = first && (q[j] != q[k]);
+    key[(size_t)t * K + k] = first ? q[k] : -1;
+  }
+}
+
+// Slots that are not the first of their (token, partition) read the row of the one that is.
+__global__ void __launch_bounds__(256) dedup_fill_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ part,
+                                                         const int32_t* __restrict__ key,
+                                                         int32_t* __restrict__ recv_row_of_slot, int N, int E, int K, int P) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= N) return;
+  for (int k = 1; k < K; ++k) {
+    if (key[(size_t)t * K + k] >= 0) continue;
+    const int q = min(max(part[min(max(idx[(size_t)t * K + k], 0), E - 1)], 0), P - 1);
+    for (int j = 0; j < k; ++j)
+      if (key[(size_t)t * K + j] == q) { recv_row_of_slot[(size_t)t * K + k] = recv_row_of_slot[(size_t)t * K + j]; break; }
+  }
+}
+
+__global__ void __launch_bounds__(256) dedup_tokens_kernel(const int32_t* __restrict__ slot_of_recv_row,
+                                                           int32_t* __restrict__ token_of_recv_row, long long cap, int K) {
+  const long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= cap) return;
+  const int s = slot_of_recv_row[r];
+  token_of_recv_row[r] = s >= 0 ? s / K : -1;
+}
+
+// Stage 1, one warp per token: the token's row is read once and written to the receive row of every
+// partition that needs it.
+template <typename T>
+__global__ void __launch_bounds__(256) dedup_send_kernel(const T* __restrict__ X, const int32_t* __restrict__ key,
+                                                         const int32_t* __restrict__ recv_row_of_slot, T* __restrict__ Xr,
+                                                         int N, int d, int K) {
+  using V = Vec16<T>;
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= N) return;  // warp-uniform
+  int my_row = -1;
+  if (lane < K && key[(size_t)t * K + lane] >= 0) my_row = recv_row_of_slot[(size_t)t * K + lane];
+  int rows[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) rows[k] = __shfl_sync(0xffffffffu, my_row, k);
+  const int chunks = d / V::N;
+  const T* src = X + (size_t)t * d;
+  for (int c = lane; c < chunks; c += 32) {
+    V v;
+    v.load(src + (size_t)c * V::N);
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+      if (k < K && rows[k] >= 0) v.store(Xr + (size_t)rows[k] * d + (size_t)c * V::N);
+  }
+}
+
+// Stage 2, one warp per row of the per-expert layout: Xp[r] = Xr[recv_row_of_slot[slot_of_row[r]]], padding rows zero.
+template <typename T>
+__global__ void __launch_bounds__(256) dedup_replicate_kernel(const T* __restrict__ Xr, const int32_t* __restrict__ slot_of_row,
+                                                              const int32_t* __restrict__ recv_row_of_slot,
+                                                              T* __restrict__ Xp, long long R, int d) {
+  using V = Vec16<T>;
+  const int lane = threadIdx.x & 31;
+  const long long r = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= R) return;  // warp-uniform
+  const int s = slot_of_row[r];
+  const int chunks = d / V::N;
+  T* dst = Xp + (size_t)r * d;
+  if (s < 0) {
+    V zero;
+    float zf[V::N] = {};
+    zero.from_float(zf);
+    for (int c = lane; c < chunks; c += 32) zero.store(dst + (size_t)c * V::N);
+    return;
+  }
+  const T* src = Xr + (size_t)recv_row_of_slot[s] * d;
+  for (int c = lane; c < chunks; c += 32) {
+    V v;
+    v.load(src + (size_t)c * V::N);
+    v.store(dst + (size_t)c * V::N);
+  }
+}
+
+static size_t align256_(size_t x) { return (x + 255) / 256 * 256; }
+
+size_t dispatch_dedup_ws_bytes(const c2r_config* cfg) {
+  const size_t nk = (size_t)cfg->N * cfg->K;
+  return align256_(permute_ws_bytes(cfg)) + 2 * align256_(sizeof(int32_t) * (nk > 0 ? nk : 1));
+}
+
+template <typename T>
+static int dispatch_dedup_impl(const c2r_config* cfg, const int32_t* idx, const int32_t* part, const int32_t* expert_rank,
+                               const T* X, int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row,
+                               int32_t* recv_counts, int32_t* recv_offsets, int32_t* recv_row_of_slot,
+                               int32_t* token_of_recv_row, T* Xr, T* Xp, int32_t* status, void* ws, cudaStream_t s) {
+  const int N = cfg->N, K = cfg->K, E = cfg->E, P = cfg->P;
+  const long long NK = (long long)N * K;
+  const long long R = permuted_rows(cfg);
+  const long long cap = (long long)N * (K < P ? K : P);  // rows the receive side can need
+  // the per-expert layout itself (counts, offsets, both row maps) is the plain dispatch's
+  int rc = permute_impl<T>(cfg, idx, expert_rank, nullptr, counts, offsets, row_of_slot, slot_of_row, nullptr, status, ws, s);
+  if (rc) return rc;
+  int32_t* block_counts = (int32_t*)ws;  // free again: the calls above are ordered on the stream
+  int32_t* key = (int32_t*)((char*)ws + align256_(permute_ws_bytes(cfg)));
+  int32_t* slot_of_recv_row = (int32_t*)((char*)key + align256_(sizeof(int32_t) * (NK > 0 ? NK : 1)));
+  const int nb = perm_blocks(cfg);
+  if (N > 0) {
+    dedup_keys_kernel<<<(N + 255) / 256, 256, 0, s>>>(idx, part, key, N, E, K, P);
+    C2R_LAUNCH_CHECK();
+    C2R_CUDA(cudaMemsetAsync(slot_of_recv_row, 0xFF, sizeof(int32_t) * NK, s));
+    perm_hist_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(key, NK, P, block_counts, status, 1);
+    C2R_LAUNCH_CHECK();
+  }
+  perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, P, nullptr, 1, recv_counts, recv_offsets);
+  C2R_LAUNCH_CHECK();
+  if (N > 0) {
+    perm_rank_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(key, NK, P, block_counts, recv_offsets, recv_row_of_slot,
+                                                    slot_of_recv_row, 1);
+    C2R_LAUNCH_CHECK();
+    dedup_fill_kernel<<<(N + 255) / 256, 256, 0, s>>>(idx, part, key, recv_row_of_slot, N, E, K, P);
+    C2R_LAUNCH_CHECK();
+    dedup_tokens_kernel<<<(int)((cap + 255) / 256), 256, 0, s>>>(slot_of_recv_row, token_of_recv_row, cap, K);
+    C2R_LAUNCH_CHECK();
+    if (X != nullptr) {
+      dedup_send_kernel<T><<<(N + 7) / 8, 256, 0, s>>>(X, key, recv_row_of_slot, Xr, N, cfg->d, K);
+      C2R_LAUNCH_CHECK();
+    }
+  }
+  if (X != nullptr && R > 0) {
+    dedup_replicate_kernel<T><<<(int)((R + 7) / 8), 256, 0, s>>>(Xr, slot_of_row, recv_row_of_slot, Xp, R, cfg->d);
+    C2R_LAUNCH_CHECK();
+  }
+  return C2R_OK;
+}
+
+}  // namespace c2r
+
+extern "C" int c2r_dispatch_dedup(const c2r_config* cfg, const int32_t* idx, const int32_t* part,
+                                  const int32_t* expert_rank, const void* X, int32_t* counts, int32_t* offsets,
+                                  int32_t* row_of_slot, int32_t* slot_of_row, int32_t* recv_counts,
+                                  int32_t* recv_offsets, int32_t* recv_row_of_slot, int32_t* token_of_recv_row,
+                                  void* Xr, void* Xp, int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(idx && part && counts && offsets && row_of_slot && slot_of_row, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(recv_counts && recv_offsets && recv_row_of_slot && token_of_recv_row, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(cfg->P >= 1 && cfg->P <= cfg->E, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!X || (Xr && Xp), C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(ws && ws_bytes >= dispatch_dedup_ws_bytes(cfg), C2R_ERR_WORKSPACE);
+  if (cfg->dtype == C2R_BF16)
+    return dispatch_dedup_impl<__nv_bfloat16>(cfg, idx, part, expert_rank, (const __nv_bfloat16*)X, counts, offsets,
+                                              row_of_slot, slot_of_row, recv_counts, recv_offsets, recv_row_of_slot,
+                                              token_of_recv_row, (__nv_bfloat16*)Xr, (__nv_bfloat16*)Xp, status, ws,
+                                              as_stream(stream));
+  return dispatch_dedup_impl<float>(cfg, idx, part, expert_rank, (const float*)X, counts, offsets, row_of_slot, slot_of_row,
+                                    recv_counts, recv_offsets, recv_row_of_slot, token_of_recv_row, (float*)Xr, (float*)Xp,
+                                    status, ws, as_stream(stream));
 }

@@ -240,3 +240,51 @@ def test_random_sets_control():
     L = G.random_logits(9, N, E)
     idx, w, _, st = _route_gpu(L, host(mask).view(np.uint64), K, T)
     assert np.array_equal(idx, O.c2r_route(L, ref, K)[0]) and st == 0
+
+
+@pytest.mark.parametrize("E,K,N,P,align", [(8, 2, 512, 2, 1), (60, 4, 16384, 4, 128), (60, 4, 3001, 8, 128), (16, 4, 130, 16, 8),
+                                           (64, 8, 77, 3, 128), (5, 1, 1, 1, 1), (12, 3, 1000, 5, 4)])
+def test_dispatch_dedup_two_stages(E, K, N, P, align):
+    """Zero-redundancy dispatch: receive-side index and both copy stages bit-exact against the oracle,
+    and the per-expert layout identical to the plain dispatch's."""
+    b = B()
+    d = 64
+    idx, _ = O.topk_route(G.random_logits(E + N + P, N, E), K)
+    rng = np.random.default_rng(E + P)
+    part = rng.integers(0, P, E)
+    part[:P] = np.arange(P)
+    rank = np.argsort(np.argsort(part * E + np.arange(E)))  # partition-major layout
+    X = G.normal(2, G.S_X, (N, d))
+    for bf16 in (False, True):
+        cfg = b.make_config(N, d, E, 16, K, K - 1, P, 0, b.BF16 if bf16 else b.F32, align)
+        R = b.permuted_rows(cfg)
+        cap = N * min(K, P)
+        Xh = G.round_bf16(X) if bf16 else X
+        Xd = dev(Xh, torch.bfloat16 if bf16 else None)
+        i32 = dict(dtype=torch.int32, device="cuda")
+        counts, offsets = torch.zeros(E, **i32), torch.zeros(E + 1, **i32)
+        ros, sor = torch.zeros(N * K, **i32), torch.zeros(R, **i32)
+        rc, ro = torch.full((P,), -9, **i32), torch.full((P + 1,), -9, **i32)
+        rrs, tok = torch.full((N * K,), -9, **i32), torch.full((cap,), -9, **i32)
+        Xr = torch.full((cap, d), 3.0, dtype=Xd.dtype, device="cuda")
+        Xp = torch.full((R, d), 3.0, dtype=Xd.dtype, device="cuda")
+        ws = torch.empty(b.workspace_bytes(cfg, b.WS_DISPATCH_DEDUP), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, **i32)
+        b.dispatch_dedup(cfg, dev(idx.astype(np.int32)), dev(part.astype(np.int32)), dev(rank.astype(np.int32)), Xd,
+                         counts, offsets, ros, sor, rc, ro, rrs, tok, Xr, Xp, status, ws)
+        c_ref, o_ref, ros_ref, sor_ref = O.permute_index(idx, E, rank, align)
+        assert np.array_equal(host(counts), c_ref) and np.array_equal(host(offsets), o_ref)
+        assert np.array_equal(host(ros), ros_ref)
+        assert np.array_equal(host(sor)[: sor_ref.size], sor_ref) and np.all(host(sor)[sor_ref.size:] == -1)
+        rc_ref, ro_ref, rrs_ref, tok_ref = O.dedup_dispatch_index(idx, part, P)
+        assert np.array_equal(host(rc), rc_ref) and np.array_equal(host(ro), ro_ref)
+        assert np.array_equal(host(rrs), rrs_ref)
+        D = int(ro_ref[P])
+        assert np.array_equal(host(tok)[:D], tok_ref) and np.all(host(tok)[D:] == -1)
+        assert D == O.dispatch_volume(idx, part, P)["dedup"]
+        Xr_ref, Xp_ref = O.dedup_dispatch(Xh, sor_ref, rrs_ref, tok_ref)
+        assert np.array_equal(host(Xr)[:D], Xr_ref)
+        ref_full = np.zeros((R, d), dtype=np.float32)
+        ref_full[: sor_ref.size] = Xp_ref
+        assert np.array_equal(host(Xp), ref_full)
+        assert int(status.item()) == 0
