@@ -231,7 +231,10 @@ int c2r_route_bwd(const c2r_config* cfg, const float* w, const float* dw, float*
 
 /* Gate weight gradients: dWg[e,:] = sum_t dL[t,e] X[t,:], evaluated over expert e's rows of Xp
  * (dl addressed through slot_of_row); dwsg[:] = sum_t dz[t] X[t,:].
- * out: dWg [E,d] float; dwsg [d] float (iff dz != NULL).  ws: C2R_WS_GATE_BWD bytes. */
+ * out: dWg [E,d] float; dwsg [d] float (iff dz != NULL).  ws: C2R_WS_GATE_BWD bytes.
+ * bf16 with X and ws given: evaluated as one tensor-core GEMM dL^T X over a dense [N,64] bf16 copy of the
+ * gradient w.r.t. the logits (dl and dz rounded to bf16, fp32 accumulation, token splits added in a fixed
+ * order); otherwise a row-serial fp32 kernel over Xp. */
 int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
                  const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
                  float* dWg, float* dwsg, void* ws, size_t ws_bytes, void* stream);

@@ -39,7 +39,7 @@ int simt_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void*
 
 // Tensor-core (tcgen05) path, bf16 only.
 enum { TC_ROWS = 0, TC_WGRAD = 1 };
-enum { TC_EPI_SWIGLU_FWD = 0, TC_EPI_F32 = 1, TC_EPI_SWIGLU_BWD = 2, TC_EPI_WGRAD_BF16 = 3 };
+enum { TC_EPI_SWIGLU_FWD = 0, TC_EPI_F32 = 1, TC_EPI_SWIGLU_BWD = 2, TC_EPI_WGRAD_BF16 = 3, TC_EPI_T_F32 = 4 };
 bool tc_supported(const c2r_config* cfg, int nE, int I, int64_t R);
 int tc_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
                   const int32_t* offsets, const void* W13p, const void* W2, void* AB, void* H, void* Yp,
@@ -56,6 +56,11 @@ int gate_tc_launch(const c2r_config* cfg, const void* X, const void* Wg, const v
 // c2r_gate_logits with a status word for the bounded waits of the tensor-core kernel.
 int gate_logits_impl(const c2r_config* cfg, const void* X, const void* Wg, const void* wsg, float* L, float* z,
                      int32_t* status, void* stream);
+
+// Gate weight gradient on the tensor cores: partial[s][c][:] = sum over the tokens of split s of dLd[t,c] X[t,:],
+// dLd [N,64] bf16 the dense gradient w.r.t. the logits (column E: shared gate), splits given by device arrays.
+int tc_gate_wgrad(const c2r_config* cfg, const void* X, const void* dLd, float* partial, int n_splits,
+                  const int32_t* split_counts, const int32_t* split_offsets, int32_t* status, cudaStream_t s);
 
 size_t permute_ws_bytes(const c2r_config* cfg);
 size_t gate_bwd_ws_bytes(const c2r_config* cfg);

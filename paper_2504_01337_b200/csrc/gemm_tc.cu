@@ -497,6 +497,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
         __syncwarp();
+      } else if (p.epi == TC_EPI_T_F32) {
+        // transposed fp32 store out[group][column][row]: a warp's 32 rows are contiguous in memory
+        float* obase = (float*)p.C + (long long)ti.expert * p.sC + mrow;
+        for (int ci = hsel; ci < (w >> 4); ci += 2) {
+          uint32_t r0[16];
+          if (have_acc) {
+            tc_ld16(taddr_row + 16 * ci, r0);
+            tc_ld_wait();
+          }
+          if (lane < rows_valid) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              obase[(long long)(TILE_N * ti.jn + 16 * ci + i) * p.ldc] = have_acc ? __uint_as_float(r0[i]) : 0.f;
+          }
+        }
       }
       if (have_acc) {
         tc_fence_before();
@@ -630,6 +645,23 @@ int tc_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* X
   if (rc) return rc;
   p.Mout = 2 * I; p.Nout = d; p.m_tiles = (2 * I + TILE_M - 1) / TILE_M; p.n_tiles = (d + TILE_N - 1) / TILE_N;
   p.C = dW13p; p.ldc = d; p.sC = (long long)2 * I * d;
+  return launch<true, true>(ma, mb, p, s);
+}
+
+int tc_gate_wgrad(const c2r_config* cfg, const void* X, const void* dLd, float* partial, int n_splits,
+                  const int32_t* split_counts, const int32_t* split_offsets, int32_t* status, cudaStream_t s) {
+  const int d = cfg->d;
+  CUtensorMap ma, mb;
+  TcParams p{};
+  p.mode = TC_WGRAD; p.epi = TC_EPI_T_F32; p.n_experts = n_splits; p.R = cfg->N; p.I = 0;
+  p.counts = split_counts; p.offsets = split_offsets; p.status = status;
+  // out^T[d, 64] = X^T dLd per split: A = X as [k = token][m = d], B = dLd as [k = token][n = 64], both MN-major
+  int rc = make_map(&ma, X, d, cfg->N, 0, 64, 64);
+  if (rc) return rc;
+  rc = make_map(&mb, dLd, 64, cfg->N, 0, 64, 64);
+  if (rc) return rc;
+  p.Mout = d; p.Nout = 64; p.m_tiles = (d + TILE_M - 1) / TILE_M; p.n_tiles = 1;
+  p.C = partial; p.ldc = d; p.sC = 64ll * d;
   return launch<true, true>(ma, mb, p, s);
 }
 

@@ -1,6 +1,7 @@
 // Dispatch on one device: atomic-free histogram / prefix-scan / stable rank over experts, the
 // 16-byte vectorised row gather, the weighted combine and their backward twins.
 #include "c2r_common.cuh"
+#include "gemm.h"
 
 namespace c2r {
 
@@ -450,7 +451,76 @@ inline int perm_blocks(const c2r_config* cfg) {
 size_t permute_ws_bytes(const c2r_config* cfg) {
   return sizeof(int32_t) * (size_t)(perm_blocks(cfg) > 0 ? perm_blocks(cfg) : 1) * cfg->E;
 }
-size_t gate_bwd_ws_bytes(const c2r_config* cfg) { return sizeof(float) * (size_t)GWS_SPLITS * cfg->d; }
+// ---- gate weight gradient as a tensor-core GEMM (bf16) -----------------------------------------
+// dWg = dL^T X with dL dense [N,64] bf16: column e holds dl of the slot routed to expert e, column E
+// the shared-gate gradient dz, everything else zero.  The token range is cut into splits that run
+// as the "groups" of the grouped GEMM; their fp32 partial results are added in split order.
+constexpr int GW_COLS = 64;
+
+struct GateWgradPlan {
+  int splits, per;                     // tokens per split (a multiple of 64)
+  size_t off_partial, off_counts, bytes;
+};
+static GateWgradPlan gate_wgrad_plan(const c2r_config* cfg) {
+  GateWgradPlan g;
+  const int m_tiles = (cfg->d + 255) / 256;
+  int splits = 64 / (m_tiles > 0 ? m_tiles : 1);
+  if (splits < 1) splits = 1;
+  int per = (cfg->N + splits - 1) / splits;
+  per = (per + 63) / 64 * 64;
+  if (per < 64) per = 64;
+  splits = cfg->N > 0 ? (cfg->N + per - 1) / per : 1;
+  g.splits = splits; g.per = per;
+  size_t o = ((size_t)(cfg->N > 0 ? cfg->N : 1) * GW_COLS * 2 + 255) / 256 * 256;
+  g.off_partial = o;
+  o += ((size_t)splits * GW_COLS * cfg->d * sizeof(float) + 255) / 256 * 256;
+  g.off_counts = o;
+  o += 256 * ((2 * (size_t)splits + 1) * sizeof(int32_t) / 256 + 1);
+  g.bytes = o;
+  return g;
+}
+
+// one block per expert: scatter the slot gradients of the expert's rows into its column of dL
+__global__ void __launch_bounds__(256) gate_dl_scatter_kernel(const int32_t* __restrict__ counts,
+                                                              const int32_t* __restrict__ offsets,
+                                                              const int32_t* __restrict__ slot_of_row,
+                                                              const float* __restrict__ dl,
+                                                              __nv_bfloat16* __restrict__ dLd, int K) {
+  const int e = blockIdx.x;
+  const int r0 = offsets[e], n = counts[e];
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int sl = slot_of_row[r0 + i];
+    if (sl >= 0) dLd[(size_t)(sl / K) * GW_COLS + e] = __float2bfloat16_rn(dl[sl]);
+  }
+}
+// shared-gate column and the split table
+__global__ void __launch_bounds__(256) gate_dz_kernel(const float* __restrict__ dz, __nv_bfloat16* __restrict__ dLd, int N,
+                                                      int E, int per, int splits, int32_t* __restrict__ split_counts,
+                                                      int32_t* __restrict__ split_offsets) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (dz != nullptr && t < N) dLd[(size_t)t * GW_COLS + E] = __float2bfloat16_rn(dz[t]);
+  if (blockIdx.x == 0 && threadIdx.x <= splits) {
+    const int lo = min(N, threadIdx.x * per);
+    split_offsets[threadIdx.x] = lo;
+    if (threadIdx.x < splits) split_counts[threadIdx.x] = min(N, lo + per) - lo;
+  }
+}
+__global__ void __launch_bounds__(256) gate_wgrad_reduce_kernel(const float* __restrict__ partial, int splits, int E, int d,
+                                                                float* __restrict__ dWg, float* __restrict__ dwsg) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  const int e = blockIdx.y;  // 0..E: row E is the shared gate
+  if (c >= d) return;
+  float acc = 0.f;
+  for (int sp = 0; sp < splits; ++sp) acc += partial[((size_t)sp * GW_COLS + e) * d + c];
+  if (e < E) dWg[(size_t)e * d + c] = acc;
+  else if (dwsg != nullptr) dwsg[c] = acc;
+}
+
+size_t gate_bwd_ws_bytes(const c2r_config* cfg) {
+  const size_t simt = sizeof(float) * (size_t)GWS_SPLITS * cfg->d;
+  const size_t tc = cfg->dtype == C2R_BF16 ? gate_wgrad_plan(cfg).bytes : 0;
+  return simt > tc ? simt : tc;
+}
 
 template <typename T>
 int permute_impl(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const T* X, int32_t* counts,
@@ -583,6 +653,25 @@ static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp,
                            const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
                            float* dWg, float* dwsg, void* ws, cudaStream_t s) {
   using V = Vec16<T>;
+  if (sizeof(T) == 2 && X != nullptr && ws != nullptr && cfg->N > 0 && cfg->d % 16 == 0 && cfg->E < GW_COLS &&
+      ((uintptr_t)X & 15u) == 0 && tc_supported(cfg, 1, 16, cfg->N)) {
+    const GateWgradPlan g = gate_wgrad_plan(cfg);
+    __nv_bfloat16* dLd = (__nv_bfloat16*)ws;
+    float* partial = (float*)((char*)ws + g.off_partial);
+    int32_t* sc = (int32_t*)((char*)ws + g.off_counts);
+    int32_t* so = sc + g.splits;
+    C2R_CUDA(cudaMemsetAsync(dLd, 0, (size_t)cfg->N * GW_COLS * 2, s));
+    gate_dl_scatter_kernel<<<cfg->E, 256, 0, s>>>(counts, offsets, slot_of_row, dl, dLd, cfg->K);
+    C2R_LAUNCH_CHECK();
+    gate_dz_kernel<<<(cfg->N + 255) / 256, 256, 0, s>>>(dz, dLd, cfg->N, cfg->E, g.per, g.splits, sc, so);
+    C2R_LAUNCH_CHECK();
+    int rc = tc_gate_wgrad(cfg, X, dLd, partial, g.splits, sc, so, nullptr, s);
+    if (rc) return rc;
+    gate_wgrad_reduce_kernel<<<dim3((cfg->d + 255) / 256, cfg->E + 1), 256, 0, s>>>(partial, g.splits, cfg->E, cfg->d,
+                                                                                   dWg, dz ? dwsg : nullptr);
+    C2R_LAUNCH_CHECK();
+    return C2R_OK;
+  }
   const int colblocks = (cfg->d + 32 * V::N - 1) / (32 * V::N);
   gate_wgrad_kernel<T><<<dim3(colblocks, cfg->E), 256, 0, s>>>((const T*)Xp, counts, offsets, slot_of_row, dl, dWg,
                                                                cfg->d);
@@ -604,6 +693,7 @@ extern "C" int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp
   C2R_REQUIRE(Xp && counts && offsets && slot_of_row && dl && dWg, C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(!dz || (X && dwsg), C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(!dz || (ws && ws_bytes >= gate_bwd_ws_bytes(cfg)), C2R_ERR_WORKSPACE);
+  if (ws && ws_bytes < gate_bwd_ws_bytes(cfg)) ws = nullptr;  // too small for the tensor-core form: row-serial kernel
   if (cfg->dtype == C2R_BF16)
     return gate_bwd_launch<__nv_bfloat16>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws,
                                           as_stream(stream));

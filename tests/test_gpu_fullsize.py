@@ -180,9 +180,11 @@ def test_fullsize_train_step(name):
     _check_expert_grads(wl, lay, X, dY, w_ref, counts, offsets, sor, experts=[int(order[0]), int(order[-1])])
     if wl.I_s:
         _check_shared_slabs(wl, lay, X, dY, slabs=[128, wl.I_s - 64] if wl.N <= 16384 else [wl.I_s - 64])
-    # any-size properties: the softmax backward gives sum_k dl[t,k] = 0, hence sum_e dWg[e,:] = 0
+    # any-size property: the softmax backward gives sum_k dl[t,k] = 0, hence sum_e dWg[e,:] = 0 -- up to the
+    # bf16 rounding of dl in the tensor-core gate gradient (2^-9 relative per term, so about 2^-9 sqrt(E) of a
+    # typical entry is left in the column sums)
     dWg = lay.host("dWg").astype(np.float64)
-    assert np.abs(dWg.sum(axis=0)).max() <= 1e-3 * np.abs(dWg).max()
+    assert np.abs(dWg.sum(axis=0)).max() <= 6 * 2.0 ** -9 * np.sqrt(wl.E) * np.sqrt(np.mean(dWg ** 2))
     for name_ in ("Y", "dX", "dW2", "dW13p"):
         assert torch.isfinite(lay.t[name_].float()).all(), name_
 
