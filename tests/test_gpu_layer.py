@@ -209,3 +209,85 @@ def test_train_step_refreshes_sets_from_live_routing():
     new_sets = O.collab_sets(Cref, wl.T)
     assert np.array_equal(lay.host("I_T"), new_sets)
     assert np.array_equal(lay.host("mask_next").view(np.uint64), mask_of(new_sets, wl.E))
+
+
+EDGE = [
+    # name,            N,   d,  E,  I,   K, T, P, I_s
+    ("tiny-dims", 70, 16, 4, 16, 2, 2, 2, 16),         # one k-block, one 16-wide N tile, ragged everything
+    ("one-token", 1, 64, 8, 144, 2, 3, 2, 0),          # most experts empty; I = 128 + 16 tail block
+    ("odd-tiles", 1500, 128, 6, 272, 3, 4, 3, 400),    # experts with odd numbers of 128-row blocks, I and I_s tails
+    ("single-expert", 300, 64, 1, 64, 1, 0, 1, 0),     # E = 1, K = 1: a dense MLP through the grouped path
+    ("wide-d", 260, 4096, 4, 48, 2, 2, 2, 0),          # 16 pair tiles along d, I < one tile
+]
+
+
+@pytest.mark.parametrize("name,N,d,E,I,K,T,P,I_s", EDGE)
+def test_edge_shapes_bf16_tensor_core_path(name, N, d, E, I, K, T, P, I_s):
+    """Shapes at the edges of the CTA-pair GEMM's tiling: tails in every dimension, empty experts,
+    a single expert, a single token."""
+    wl = G.Workload(name, N=N, d=d, E=E, I=I, K=K, T=T, P=P, I_s=I_s, bf16=True, seed=23)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    sh = G.shared_weights(wl) if I_s else None
+    sets = random_sets(E, T, seed=2) if T > 0 else np.zeros((E, 0), dtype=np.int64)
+    lay = _layer(wl, backward=True)
+    lay.set_params(Wg, W1, W3, W2, wsg, sh)
+    lay.set_routing(mask=mask_of(sets, E) if T > 0 else None)
+    lay.set_input(X, dY)
+    lay.forward()
+    lay.backward()
+    torch.cuda.synchronize()
+    assert int(lay.t["status"].item()) == 0
+    Lg = lay.host("L")
+    f = O.layer_fwd(X, Wg, W1, W3, W2, sets if T > 0 else None, K, row_align=lay.cfg.row_align, shared=sh, wsg=wsg, logits=Lg)
+    assert np.array_equal(lay.host("idx"), f["idx"])
+    live = live_rows(f["counts"], f["offsets"])
+    assert_close_elem(lay.host("H")[live], f["H"][live], what="H")
+    assert_close_rms(lay.host("Y"), f["Y"], 2e-2, "Y")
+    f2 = O.layer_fwd(X, Wg, W1, W3, W2, sets if T > 0 else None, K, row_align=lay.cfg.row_align, shared=sh, wsg=wsg)
+    if not np.array_equal(f2["idx"], f["idx"]):
+        pytest.skip("fp32 and fp64 logits disagree on a near-tie; backward parity needs equal routing")
+    g = O.layer_bwd(X, Wg, W1, W3, W2, f2, dY, shared=sh, wsg=wsg)
+    grads = [host(t) for t in lay.unpacked_grads()]
+    # These shapes probe indexing, not precision: with a handful of rows per expert (or a contraction of 96
+    # terms) a gradient element is a sum of few products whose operands each went through up to three bf16
+    # roundings, so the per-element allowance is four half-ulps of the reference (three operand roundings and
+    # the result's own) on top of 3e-2 * RMS; the tensor-level RMS bound is relaxed to 1e-2 likewise.
+    # (a single token makes every gradient element ONE product, with no averaging at all: 6e-2 there)
+    edge = dict(frac=6e-2 if N < 8 else 3e-2, ulps=4.0, rms_frac=1e-2)
+    for e in range(E):  # per expert, so that experts without tokens (exact zeros) do not deflate the RMS
+        for got, ref, nm in ((grads[0][e], g["dW1"][e], "dW1"), (grads[1][e], g["dW3"][e], "dW3"),
+                             (lay.host("dW2")[e], g["dW2"][e], "dW2")):
+            if f["counts"][e] == 0:
+                assert not got.any(), f"{nm}[{e}] of an expert without tokens"
+            else:
+                assert_close_rms(got, ref, what=f"{nm}[{e}]", **edge)
+    assert_close_rms(lay.host("dX"), g["dX"], what="dX", **edge)
+    assert_close_rms(lay.host("dWg"), g["dWg"], what="dWg", **edge)  # dl enters the gate GEMM rounded to bf16
+    if I_s:
+        assert_close_rms(grads[2], g["dWs1"], 2e-2, "dWs1")
+        assert_close_rms(lay.host("dWs2")[0], g["dWs2"], 2e-2, "dWs2")
+        assert_close_rms(lay.host("dwsg"), g["dwsg"], 2e-2, "dwsg", out_bf16=False)
+
+
+def test_weight_gradients_accumulate():
+    """accumulate != 0 adds the new weight gradients to what the buffers hold (bf16 read-modify-write)."""
+    wl = G.Workload("acc", N=600, d=128, E=4, I=144, K=2, T=2, P=2, I_s=64, bf16=True, seed=4)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    lay = _layer(wl, backward=True)
+    lay.set_params(Wg, W1, W3, W2, wsg, G.shared_weights(wl))
+    lay.set_routing(mask=mask_of(random_sets(wl.E, wl.T, seed=1), wl.E))
+    lay.set_input(X, dY)
+    lay.forward()
+    lay.backward()
+    torch.cuda.synchronize()
+    once = {k: lay.t[k].float().clone() for k in ("dW13p", "dW2", "dWs13p", "dWs2")}
+    lay.backward(accumulate=True)
+    torch.cuda.synchronize()
+    for k, v in once.items():
+        twice = lay.t[k].float()
+        # 2x is exact in bf16 up to the rounding of the sum: within one bf16 ulp of 2v
+        assert torch.all((twice - 2 * v).abs() <= 2.0 ** -7 * (2 * v).abs() + 1e-30), k

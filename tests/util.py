@@ -17,7 +17,7 @@ def host(t):
     return (t.float() if t.dtype == torch.bfloat16 else t).cpu().numpy()
 
 
-def assert_close_rms(got, ref, frac=2e-2, what="", out_bf16=True, rms_frac=5e-3):
+def assert_close_rms(got, ref, frac=2e-2, what="", out_bf16=True, rms_frac=5e-3, ulps=1.0):
     """bf16 bar.  Every element: |err| <= frac * RMS(ref) + 2^-8 |ref|, where the second term is the
     representation error of a bf16-stored result (half an ulp, which no implementation can avoid;
     dropped with out_bf16=False for results stored in fp32).  And over the tensor:
@@ -29,7 +29,7 @@ def assert_close_rms(got, ref, frac=2e-2, what="", out_bf16=True, rms_frac=5e-3)
         return
     rms = float(np.sqrt(np.mean(ref ** 2)))
     err = np.abs(got - ref)
-    tol = frac * rms + (2.0 ** -8 * np.abs(ref) if out_bf16 else 0.0)
+    tol = frac * rms + (ulps * 2.0 ** -8 * np.abs(ref) if out_bf16 else 0.0)
     worst = float(np.max(err - tol))
     assert worst <= 0.0, f"{what}: max|err|={err.max():.3e} ({err.max() / rms:.4f} RMS), over tolerance by {worst:.3e}"
     erms = float(np.sqrt(np.mean(err ** 2)))
