@@ -288,3 +288,24 @@ def test_dispatch_dedup_two_stages(E, K, N, P, align):
         ref_full[: sor_ref.size] = Xp_ref
         assert np.array_equal(host(Xp), ref_full)
         assert int(status.item()) == 0
+
+
+def test_T_P_sweep_report_matches_oracle():
+    """The sweep utility's numbers are the oracle's: T = E-1 reproduces conventional Top-K (Fig. 3's
+    degenerate case), and a constrained point matches routing, volume, load and Eq. 3 computed on the CPU."""
+    from paper_2504_01337_b200 import report
+    wl = G.Workload("sweep", N=3000, d=64, E=16, I=16, K=4, T=6, P=4, bf16=False, n_calib=2000, seed=8, skew=True)
+    rep = report.sweep(wl, Ts=[3, 6, 15], Ps=[2, 4])
+    assert rep["T"][15] == rep["topk"]
+    L, Lc = G.skewed_logits(wl), G.skewed_logits(wl, calib=True)
+    Cc = O.collab_count(O.topk_route(Lc, wl.K)[0], wl.E)
+    sets = O.collab_sets(Cc, 6)
+    idx, _ = O.c2r_route(L, sets, wl.K)
+    got = rep["T"][6]
+    ls = O.load_stats(np.bincount(idx.reshape(-1), minlength=wl.E))
+    assert abs(got["load_max_over_mean"] - ls["max_over_mean"]) < 1e-9 and abs(got["load_cv"] - ls["cv"]) < 1e-9
+    assert abs(got["collab_degree_mean"] - O.collab_degree(O.collab_count(idx, wl.E))[1]) < 1e-4
+    for P in (2, 4):
+        v = O.dispatch_volume(idx, O.place_experts(Cc, P)[0], P)
+        assert (got[f"P{P}"]["naive"], got[f"P{P}"]["dedup"], got[f"P{P}"]["naive_cross"], got[f"P{P}"]["dedup_cross"]) == \
+               (v["naive"], v["dedup"], v["naive_x"], v["dedup_x"])
