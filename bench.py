@@ -365,9 +365,9 @@ def run_reference(args, wl):
 
 
 # DRAM bytes per launch of tc_gemm_kernel (dram__bytes_read.sum + dram__bytes_write.sum averaged over
-# the 12 launches of a step) from the ncu launch list of this very command, summarised under
+# the 12 expert-GEMM launches of a step) from the ncu launch list of this very command, summarised under
 # profiles/.  Keyed by workload; None where no capture of the current kernel exists.
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = {"c3": 1.015e9}
+GEMM_TRAFFIC_BYTES_PER_LAUNCH = {"c3": 1.035e9}
 
 
 def main():

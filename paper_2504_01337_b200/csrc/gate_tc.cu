@@ -169,13 +169,19 @@ int gate_tc_launch(const c2r_config* cfg, const void* X, const void* Wg, const v
   rc = make_map(&ms, wsg ? wsg : Wg, cfg->d, 1, 0, BK, 16);
   if (rc) return rc;
   constexpr int smem = GT_STAGES * GT_STAGE_BYTES + 1024;
-  static bool configured = false;
-  if (!configured) {
+  constexpr int MAX_DEV = 64;
+  static int sms_of_device[MAX_DEV] = {};  // SM count, also "the kernel's shared-memory limit is set on this device"
+  int dev = 0;
+  C2R_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= MAX_DEV) return C2R_ERR_UNSUPPORTED_SHAPE;
+  int sms = __atomic_load_n(&sms_of_device[dev], __ATOMIC_ACQUIRE);
+  if (sms == 0) {
     C2R_CUDA(cudaFuncSetAttribute(gate_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    configured = true;
+    C2R_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    __atomic_store_n(&sms_of_device[dev], sms, __ATOMIC_RELEASE);
   }
   const int tiles = (cfg->N + BM - 1) / BM;
-  const int grid = tiles < sm_count() ? tiles : sm_count();
+  const int grid = tiles < sms ? tiles : sms;
   gate_tc_kernel<<<grid, GT_THREADS, smem, s>>>(mx, mw, ms, L, z, cfg->N, cfg->d, cfg->E, wsg != nullptr, status);
   C2R_LAUNCH_CHECK();
   return C2R_OK;

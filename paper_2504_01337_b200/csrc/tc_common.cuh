@@ -204,14 +204,5 @@ inline int make_map(CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, 
   return C2R_OK;
 }
 
-inline int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      n = 148;
-  }
-  return n;
-}
 
 }  // namespace c2r
