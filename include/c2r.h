@@ -190,7 +190,8 @@ int c2r_unpack_weights(const c2r_config* cfg, int n_experts, int I, const void* 
  * Xp [R,d] T; counts [n_experts], offsets [n_experts+1] int32 (device); W13p packed (above);
  * W2 [n_experts, d, I] T.  out: AB [R, 2I] T (what the backward pass needs from A and B, in the
  * packed column layout: the local derivatives dH/dA = B silu'(A) in the gate columns and
- * dH/dB = silu(A) in the up columns), H [R,I] T, Yp [R,d] float.
+ * dH/dB = silu(A) in the up columns; AB == NULL skips it: forward only, e.g. inference),
+ * H [R,I] T, Yp [R,d] float.
  * R = rows of the buffers.  Padding rows of Xp must be zero.  n_experts = 1 with counts = {R},
  * offsets = {0,R} evaluates the dense shared expert.
  * bf16 runs on the tensor cores (tcgen05) when d % 16 == 0 and, for n_experts > 1, row_align is a
@@ -282,7 +283,7 @@ typedef struct c2r_layer_buffers {
   int32_t* row_of_slot; /* [N*K] */
   int32_t* slot_of_row; /* [R] */
   void* Xp;             /* [R,d] */
-  void* AB;             /* [R,2I] */
+  void* AB;             /* [R,2I]; NULL (with ABs) when no backward pass follows */
   void* H;              /* [R,I] */
   void* Yp;             /* [R,d] float */
   void* ABs;            /* [N,2I_s] */

@@ -80,10 +80,8 @@ extern "C" int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int 
   if (R == 0) return C2R_OK;
   cudaStream_t s = as_stream(stream);
   if (cfg->dtype == C2R_F32) {
-    C2R_REQUIRE(AB, C2R_ERR_INVALID_ARG);
     return simt_swiglu_fwd<float>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, s);
   }
-  C2R_REQUIRE(AB, C2R_ERR_INVALID_ARG);
   if (tc_supported(cfg, n_experts, I, R))
     return tc_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, status, s);
   return simt_swiglu_fwd<__nv_bfloat16>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, s);
@@ -124,7 +122,7 @@ extern "C" int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
   const bool shared = cfg->I_s > 0;
   C2R_REQUIRE(b->ws && b->ws_bytes >= c2r_workspace_bytes(cfg, C2R_WS_LAYER), C2R_ERR_WORKSPACE);
   if (shared)
-    C2R_REQUIRE(b->wsg && b->z && b->Ws13p && b->Ws2 && b->ABs && b->Hs && b->Ys && b->s_counts && b->s_offsets,
+    C2R_REQUIRE(b->wsg && b->z && b->Ws13p && b->Ws2 && b->Hs && b->Ys && b->s_counts && b->s_offsets,
                 C2R_ERR_INVALID_ARG);
   const int64_t R = permuted_rows(cfg);
   C2R_TRY(gate_logits_impl(cfg, b->X, b->Wg, shared ? b->wsg : nullptr, b->L, b->z, b->status, stream));

@@ -136,9 +136,11 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(SimtGemm g) {
         const float b = acc2[i][j];
         const float sg = 1.0f / (1.0f + expf(-v));
         const float as = v * sg;
-        T* sv = (T*)g.C + (long long)(r0 + m) * 2 * g.I;
-        sv[pg] = from_f32<T>(b * (sg + as - as * sg));
-        sv[pu] = from_f32<T>(as);
+        if (g.C != nullptr) {  // inference: nothing is kept for a backward pass
+          T* sv = (T*)g.C + (long long)(r0 + m) * 2 * g.I;
+          sv[pg] = from_f32<T>(b * (sg + as - as * sg));
+          sv[pu] = from_f32<T>(as);
+        }
         ((T*)g.aux_out)[(long long)(r0 + m) * g.I + n] = from_f32<T>(as * b);
       } else {  // SIMT_EPI_SWIGLU_BWD: v = dH[r, n]; dA = dH * (dH/dA), dB = dH * (dH/dB) at the packed columns
         const int pg = pack_col(n, g.I), pu = pg + pack_width(n, g.I);

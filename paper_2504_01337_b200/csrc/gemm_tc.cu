@@ -395,6 +395,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int g = hsel; g < n_groups; g += 2) {
           const int c = 64 * g;
           const int vbytes = 2 * min(64, w - c);
+          const bool keep = p.C != nullptr;  // false: inference, only H is produced
           uint4 up[8];
 #pragma unroll
           for (int pc = 0; pc < 4; ++pc) {
@@ -416,23 +417,27 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               ga[i] = b * (sg + as - as * sg);     // b silu'(a), silu'(a) = s (1 + a (1 - s))
               gb[i] = as;
             }
-            sts128(stg_addr(buf0, lane, 2 * pc), pack_bf16x8(ga)); sts128(stg_addr(buf0, lane, 2 * pc + 1), pack_bf16x8(ga + 8));
             sts128(stg_addr(buf1, lane, 2 * pc), pack_bf16x8(h)); sts128(stg_addr(buf1, lane, 2 * pc + 1), pack_bf16x8(h + 8));
-            up[2 * pc] = pack_bf16x8(gb); up[2 * pc + 1] = pack_bf16x8(gb + 8);
+            if (keep) {
+              sts128(stg_addr(buf0, lane, 2 * pc), pack_bf16x8(ga)); sts128(stg_addr(buf0, lane, 2 * pc + 1), pack_bf16x8(ga + 8));
+              up[2 * pc] = pack_bf16x8(gb); up[2 * pc + 1] = pack_bf16x8(gb + 8);
+            }
           }
           __syncwarp();
           uint8_t* gab = (uint8_t*)p.C + row0 * (4ll * p.I) + 2 * (256 * ti.jn + c);
-          stage_to_global(buf0, gab, 4ll * p.I, rows_valid, vbytes, lane);
+          if (keep) stage_to_global(buf0, gab, 4ll * p.I, rows_valid, vbytes, lane);
           stage_to_global(buf1, (uint8_t*)p.H + row0 * (2ll * p.I) + 2 * (128 * ti.jn + c), 2ll * p.I, rows_valid, vbytes, lane);
           __syncwarp();
+          if (keep) {
 #pragma unroll
-          for (int pc = 0; pc < 4; ++pc) {
-            if (32 * pc >= vbytes) break;
-            sts128(stg_addr(buf0, lane, 2 * pc), up[2 * pc]); sts128(stg_addr(buf0, lane, 2 * pc + 1), up[2 * pc + 1]);
+            for (int pc = 0; pc < 4; ++pc) {
+              if (32 * pc >= vbytes) break;
+              sts128(stg_addr(buf0, lane, 2 * pc), up[2 * pc]); sts128(stg_addr(buf0, lane, 2 * pc + 1), up[2 * pc + 1]);
+            }
+            __syncwarp();
+            stage_to_global(buf0, gab + 2 * w, 4ll * p.I, rows_valid, vbytes, lane);
+            __syncwarp();
           }
-          __syncwarp();
-          stage_to_global(buf0, gab + 2 * w, 4ll * p.I, rows_valid, vbytes, lane);
-          __syncwarp();
         }
       } else if (p.epi == TC_EPI_F32) {
         const int n_groups = (w + 31) >> 5;  // 32 fp32 columns = 128 bytes

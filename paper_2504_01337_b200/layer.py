@@ -45,7 +45,6 @@ class C2RLayer:
         t["row_of_slot"] = buf((N * K,), i32)
         t["slot_of_row"] = buf((R,), i32)
         t["Xp"] = buf((R, d))
-        t["AB"] = buf((R, 2 * I))
         t["H"] = buf((R, I))
         t["Yp"] = buf((R, d), f32)
         t["Y"] = buf((N, d))
@@ -54,12 +53,14 @@ class C2RLayer:
         t["ws"] = torch.empty((B.workspace_bytes(self.cfg, B.WS_LAYER),), dtype=torch.uint8, device=dev)
         if I_s:
             t["z"] = buf((N,), f32)
-            t["ABs"] = buf((N, 2 * I_s))
             t["Hs"] = buf((N, I_s))
             t["Ys"] = buf((N, d), f32)
             t["s_counts"] = torch.tensor([N], dtype=i32, device=dev)
             t["s_offsets"] = torch.tensor([0, N], dtype=i32, device=dev)
         if backward:
+            t["AB"] = buf((R, 2 * I))  # what the backward pass needs from the up-projection
+            if I_s:
+                t["ABs"] = buf((N, 2 * I_s))
             t["dY"] = buf((N, d))
             t["dYp"] = buf((R, d))
             t["dAB"] = buf((R, 2 * I))

@@ -255,8 +255,8 @@ def test_c4_skewed_routing_topk_vs_c2r_and_forward():
     rank_d = torch.from_numpy(rank_ref.astype(np.int32)).cuda()
     b.gate_logits(cfg, t["X"], t["Wg"], t["wsg"], t["L"], t["z"])  # only z (the shared-expert gate) is used from this call
     b.permute(cfg, idx, rank_d, t["X"], t["counts"], t["offsets"], t["row_of_slot"], t["slot_of_row"], t["Xp"], status, ws)
-    b.grouped_swiglu_fwd(cfg, E, wl.I, lay.R, t["Xp"], t["counts"], t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["Yp"], status)
-    b.grouped_swiglu_fwd(cfg, 1, wl.I_s, N, t["X"], t["s_counts"], t["s_offsets"], t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["Ys"], status)
+    b.grouped_swiglu_fwd(cfg, E, wl.I, lay.R, t["Xp"], t["counts"], t["offsets"], t["W13p"], t["W2"], t.get("AB"), t["H"], t["Yp"], status)
+    b.grouped_swiglu_fwd(cfg, 1, wl.I_s, N, t["X"], t["s_counts"], t["s_offsets"], t["Ws13p"], t["Ws2"], t.get("ABs"), t["Hs"], t["Ys"], status)
     b.combine(cfg, t["Yp"], w, t["row_of_slot"], t["Ys"], t["z"], t["Y"])
     torch.cuda.synchronize()
     assert int(status.item()) == 0
