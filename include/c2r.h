@@ -123,7 +123,8 @@ int c2r_place_experts(const c2r_config* cfg, const int32_t* C_host, int mode, in
  * expert_rank[idx[s]] (NULL = identity), then the row gather.
  * out: counts [E] int32; offsets [E+1] int32 (start row of expert e, a multiple of row_align;
  * offsets[E] = end of the layout); row_of_slot [N*K] int32; slot_of_row [c2r_permuted_rows] int32
- * (-1 = padding); Xp [c2r_permuted_rows, d] T with Xp[r,:] = X[slot_of_row[r]/K,:], padding rows zero.
+ * (-1 = padding); Xp [c2r_permuted_rows, d] T with Xp[r,:] = X[slot_of_row[r]/K,:]; the padding rows that
+ * close an expert's aligned segment are zero, rows at or beyond offsets[E] are not written.
  * X == NULL builds the index only.  Atomic-free and deterministic.
  * ws: C2R_WS_PERMUTE bytes.  status as in c2r_route. */
 int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,

@@ -142,13 +142,118 @@ __global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_kernel(const int32_
   }
 }
 
-// Row gather, one warp per token: the token's row is read once and written to its K rows.
+// The scan folded into the rank pass (for batches of at most PERM_FUSED_MAX_BLOCKS blocks): every block
+// adds up the histogram rows of the blocks before it and of all blocks (E columns, coalesced), derives the
+// aligned segment offsets itself, and block 0 publishes counts and offsets.  One launch and one
+// dependent round trip fewer than hist -> scan -> rank.
+constexpr int PERM_FUSED_MAX_BLOCKS = 1024;
+__global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_fused_kernel(const int32_t* __restrict__ idx, long long NK, int E,
+                                                                          const int32_t* __restrict__ block_counts,
+                                                                          int n_blocks,
+                                                                          const int32_t* __restrict__ expert_rank,
+                                                                          int row_align, int32_t* __restrict__ counts,
+                                                                          int32_t* __restrict__ offsets,
+                                                                          int32_t* __restrict__ row_of_slot,
+                                                                          int32_t* __restrict__ slot_of_row) {
+  __shared__ int warp_cnt[PERM_WARPS][64];
+  __shared__ int s_before[64], s_total[64], s_by_rank[64], s_off[65];
+  __shared__ int s_part[2][PERM_WARPS * 32 / 64][64];  // partial sums: [before | total][quarter of the blocks][expert]
+  for (int i = threadIdx.x; i < PERM_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
+  {
+    constexpr int PARTS = PERM_WARPS * 32 / 64;
+    const int e = threadIdx.x & 63, part = threadIdx.x >> 6;
+    int before = 0, total = 0;
+    if (e < E) {
+#pragma unroll 8
+      for (int b = part; b < n_blocks; b += PARTS) {
+        const int v = block_counts[(size_t)b * E + e];
+        total += v;
+        before += (b < (int)blockIdx.x) ? v : 0;
+      }
+    }
+    s_part[0][part][e] = before;
+    s_part[1][part][e] = total;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    int before = 0, total = 0;
+#pragma unroll
+    for (int q = 0; q < PERM_WARPS * 32 / 64; ++q) { before += s_part[0][q][e]; total += s_part[1][q][e]; }
+    s_before[e] = before;
+    s_total[e] = total;
+    int r = expert_rank ? expert_rank[e] : e;
+    s_by_rank[min(max(r, 0), E - 1)] = e;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int cursor = 0;
+    for (int r = 0; r < E; ++r) {
+      const int e = s_by_rank[r];
+      s_off[e] = cursor;
+      cursor += (s_total[e] + row_align - 1) / row_align * row_align;
+    }
+    s_off[E] = cursor;
+  }
+  int e_reg[PERM_ITERS];
+  int flags = 0;
+  warp_count(idx, NK, E, warp_cnt, e_reg, flags, 0);
+  __syncthreads();
+  if (blockIdx.x == 0) {
+    for (int e = threadIdx.x; e <= E; e += blockDim.x) {
+      offsets[e] = s_off[e];
+      if (e < E) counts[e] = s_total[e];
+    }
+  }
+  for (int e = threadIdx.x; e < E; e += blockDim.x) {
+    int run = s_off[e] + s_before[e];
+#pragma unroll
+    for (int w = 0; w < PERM_WARPS; ++w) {
+      const int c = warp_cnt[w][e];
+      warp_cnt[w][e] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const long long base = (long long)blockIdx.x * PERM_BLOCK_SLOTS + (long long)w * PERM_ITERS * 32;
+#pragma unroll
+  for (int it = 0; it < PERM_ITERS; ++it) {
+    const long long s = base + it * 32 + lane;
+    const int e = e_reg[it];
+    const uint32_t peers = __match_any_sync(0xffffffffu, e);
+    const int start = (e >= 0) ? warp_cnt[w][e] : 0;
+    __syncwarp();
+    if (e >= 0 && lane == __ffs(peers) - 1) warp_cnt[w][e] = start + __popc(peers);
+    __syncwarp();
+    if (e >= 0) {
+      const int row = start + __popc(peers & lanemask_lt());
+      row_of_slot[s] = row;
+      slot_of_row[row] = (int32_t)s;
+    }
+  }
+}
+
+// Row gather, one warp per token: the token's row is read once and written to its K rows.  Blocks past the
+// token blocks zero the padding rows that close each expert's aligned segment (block j: expert j).
 template <typename T>
 __global__ void __launch_bounds__(256) permute_rows_kernel(const T* __restrict__ X,
                                                            const int32_t* __restrict__ row_of_slot, T* __restrict__ Xp,
-                                                           int N, int d, int K) {
+                                                           int N, int d, int K, const int32_t* __restrict__ counts,
+                                                           const int32_t* __restrict__ offsets, int token_blocks,
+                                                           int row_align) {
   using V = Vec16<T>;
   const int lane = threadIdx.x & 31;
+  if ((int)blockIdx.x >= token_blocks) {
+    const int e = blockIdx.x - token_blocks;
+    const int n = counts[e];
+    const int r0 = offsets[e] + n, r1 = offsets[e] + (n + row_align - 1) / row_align * row_align;
+    V zero;
+    float zf[V::N] = {};
+    zero.from_float(zf);
+    for (int r = r0 + (threadIdx.x >> 5); r < r1; r += blockDim.x >> 5)
+      for (int c = lane; c < d / V::N; c += 32) zero.store(Xp + (size_t)r * d + (size_t)c * V::N);
+    return;
+  }
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (t >= N) return;  // warp-uniform
   const int my_row = (lane < K) ? row_of_slot[(size_t)t * K + lane] : 0;
@@ -535,24 +640,29 @@ int permute_impl(const c2r_config* cfg, const int32_t* idx, const int32_t* exper
     perm_hist_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, status, 0);
     C2R_LAUNCH_CHECK();
   }
-  perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, cfg->E, expert_rank, cfg->row_align, counts, offsets);
-  C2R_LAUNCH_CHECK();
-  if (nb > 0) {
-    perm_rank_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, offsets, row_of_slot, slot_of_row, 0);
+  if (nb > 0 && nb <= PERM_FUSED_MAX_BLOCKS) {
+    perm_rank_fused_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, nb, expert_rank, cfg->row_align,
+                                                          counts, offsets, row_of_slot, slot_of_row);
     C2R_LAUNCH_CHECK();
+  } else {
+    perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, cfg->E, expert_rank, cfg->row_align, counts, offsets);
+    C2R_LAUNCH_CHECK();
+    if (nb > 0) {
+      perm_rank_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, offsets, row_of_slot, slot_of_row, 0);
+      C2R_LAUNCH_CHECK();
+    }
   }
   if (X != nullptr) {
-    if (cfg->N > 0) {
-      permute_rows_kernel<T><<<(cfg->N + 7) / 8, 256, 0, s>>>(X, row_of_slot, Xp, cfg->N, cfg->d, cfg->K);
-      C2R_LAUNCH_CHECK();
-    }
-    if (R > NK) {
-      int blocks = (int)((R + 7) / 8);
-      if (blocks > 1184) blocks = 1184;
-      zero_pad_rows_kernel<T><<<blocks, 256, 0, s>>>(slot_of_row, Xp, R, cfg->d);
+    // the gather, plus one block per expert that zeroes the padding rows closing its aligned segment
+    const int token_blocks = (cfg->N + 7) / 8;
+    const int pad_blocks = cfg->row_align > 1 ? cfg->E : 0;
+    if (token_blocks + pad_blocks > 0) {
+      permute_rows_kernel<T><<<token_blocks + pad_blocks, 256, 0, s>>>(X, row_of_slot, Xp, cfg->N, cfg->d, cfg->K, counts,
+                                                                    offsets, token_blocks, cfg->row_align);
       C2R_LAUNCH_CHECK();
     }
   }
+  (void)R;
   return C2R_OK;
 }
 
