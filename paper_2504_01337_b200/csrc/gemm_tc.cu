@@ -10,7 +10,8 @@
 //
 // Warp roles (320 threads per CTA): warp 0 = TMA producer (both CTAs, each for its own halves),
 // warp 1 = MMA issuer (even CTA only; owns the TMEM allocation in both), warps 2..9 = epilogue
-// (TMEM -> registers -> global, fused SwiGLU forms; two warps per TMEM lane quarter).
+// (TMEM -> registers -> a per-warp staging tile in shared memory -> global, row-contiguously; fused
+// SwiGLU forms; two warps per TMEM lane quarter).
 // Pipelines: 5 shared-memory stages (full barrier in the even CTA counts both CTAs' bytes; the
 // MMA's commit frees the stage in both CTAs) and two TMEM accumulators of 256 columns, so the
 // epilogue of tile i overlaps the MMAs of tile i+1.  Every wait is bounded: on expiry the kernel
