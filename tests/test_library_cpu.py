@@ -78,3 +78,16 @@ def test_binding_refuses_to_import_without_library(tmp_path):
             "try:\n    spec.loader.exec_module(m)\nexcept ImportError as e:\n    print('REFUSED'); sys.exit(0)\nsys.exit(1)\n")
     out = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True)
     assert out.returncode == 0 and "REFUSED" in out.stdout
+
+
+def test_bench_accounting_matches_the_workload_arithmetic():
+    """The numerators bench.py divides by measured time: algorithmic expert-GEMM flops per token
+    (forward + backward = 3 x forward, padding not counted) for the three benchmark workloads."""
+    import bench
+    c3, c2, c5 = G.WORKLOADS["c3"], G.WORKLOADS["c2"], G.WORKLOADS["c5"]
+    fwd_c3 = 6 * 4 * 2048 * 1408 + 6 * 2048 * 5632          # routed (K = 4) + shared expert
+    assert bench.flops_per_token(c3) == 3 * fwd_c3 == 415_236_096
+    assert bench.flops_per_token(c5) == bench.flops_per_token(c3)
+    assert bench.flops_per_token(c2) == 3 * 6 * 4 * 4096 * 688
+    # whole step at c3: 6.80 TFLOP, the figure the roofline line reports per 12 launches
+    assert abs(bench.flops_per_token(c3) * c3.N / 1e12 - 6.803) < 1e-3
