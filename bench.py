@@ -106,7 +106,7 @@ class ClockSampler:
                 "samples": len(sm), "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons)}
 
 
-def build_layer(wl, device, profile=True, keep=False):
+def build_layer(wl, device, profile=True, keep=False, gather_fused=False):
     """Seeded synthetic layer of workload `wl` on `device`, routed with collaborator sets profiled
     from a calibration batch by the library itself (Eq. 2 / Eq. 4) and placed by co-activation.
     keep=True also returns the calibration state (device logits, routing, C, I_T, placement)."""
@@ -116,7 +116,7 @@ def build_layer(wl, device, profile=True, keep=False):
     from paper_2504_01337_b200.layer import C2RLayer, to_device
 
     lay = C2RLayer(wl.N, wl.d, wl.E, wl.I, wl.K, wl.T, wl.P, wl.I_s, wl.bf16, backward=True, profile=profile,
-                   device=device)
+                   device=device, gather_fused=gather_fused)
     Wg, wsg = G.gate_weights(wl)
     W1, W3, W2 = G.expert_weights(wl)
     lay.set_params(Wg, W1, W3, W2, wsg, G.shared_weights(wl))
@@ -153,16 +153,20 @@ def breakdown(lay, reps=3):
     from paper_2504_01337_b200 import binding as B
     c, t = lay.cfg, lay.t
     shared = c.I_s > 0
+    fused = bool(c.flags & B.FLAG_GATHER_FUSED) and "Xp" not in t
     R = lay.R
     P = c.P
     ws = t["ws"]
     calls = [
         ("gate_logits", lambda: B.gate_logits(c, t["X"], t["Wg"], t.get("wsg"), t["L"], t.get("z"))),
         ("route", lambda: B.route(c, t["L"], t.get("mask"), t["idx"], t["w"], None, t["status"])),
-        ("permute", lambda: B.permute(c, t["idx"], t.get("expert_rank"), t["X"], t["counts"], t["offsets"],
-                                      t["row_of_slot"], t["slot_of_row"], t["Xp"], t["status"], ws)),
-        ("swiglu_fwd", lambda: B.grouped_swiglu_fwd(c, c.E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"],
-                                                    t["W2"], t["AB"], t["H"], t["Yp"])),
+        ("permute", lambda: B.permute(c, t["idx"], t.get("expert_rank"), None if fused else t["X"], t["counts"],
+                                      t["offsets"], t["row_of_slot"], t["slot_of_row"], t.get("Xp"), t["status"], ws)),
+        ("swiglu_fwd", (lambda: B.grouped_swiglu_fwd_gather(c, c.E, c.I, R, t["X"], t["slot_of_row"], t["counts"],
+                                                            t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["Yp"]))
+         if fused else
+         (lambda: B.grouped_swiglu_fwd(c, c.E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"],
+                                       t["W2"], t["AB"], t["H"], t["Yp"]))),
     ]
     if shared:
         calls.append(("shared_fwd", lambda: B.grouped_swiglu_fwd(c, 1, c.I_s, c.N, t["X"], t["s_counts"], t["s_offsets"],
@@ -173,9 +177,13 @@ def breakdown(lay, reps=3):
                                                       t["volume"][4 + P * P:])),
         ("combine_bwd", lambda: B.combine_bwd(c, t["dY"], t["Yp"], t["w"], t["row_of_slot"], t["slot_of_row"],
                                               t.get("Ys"), t.get("z"), t["dYp"], t["dw"], t.get("dYs"), t.get("dz"))),
-        ("swiglu_bwd", lambda: B.grouped_swiglu_bwd(c, c.E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"],
-                                                    t["W2"], t["AB"], t["H"], t["dYp"], t["dAB"], t["dXp"],
-                                                    t["dW13p"], t["dW2"])),
+        ("swiglu_bwd", (lambda: B.grouped_swiglu_bwd_gather(c, c.E, c.I, R, t["X"], t["slot_of_row"], t["counts"],
+                                                            t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["dYp"],
+                                                            t["dAB"], t["dXp"], t["dW13p"], t["dW2"]))
+         if fused else
+         (lambda: B.grouped_swiglu_bwd(c, c.E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"],
+                                       t["W2"], t["AB"], t["H"], t["dYp"], t["dAB"], t["dXp"],
+                                       t["dW13p"], t["dW2"]))),
     ]
     if shared:
         calls.append(("shared_bwd", lambda: B.grouped_swiglu_bwd(c, 1, c.I_s, c.N, t["X"], t["s_counts"], t["s_offsets"],
@@ -183,7 +191,7 @@ def breakdown(lay, reps=3):
                                                                  t["dABs"], t["dXs"], t["dWs13p"], t["dWs2"])))
     calls += [
         ("route_bwd", lambda: B.route_bwd(c, t["w"], t["dw"], t["dl"])),
-        ("gate_bwd", lambda: B.gate_bwd(c, t["X"], t["Xp"], t["counts"], t["offsets"], t["slot_of_row"], t["dl"],
+        ("gate_bwd", lambda: B.gate_bwd(c, t["X"], t.get("Xp"), t["counts"], t["offsets"], t["slot_of_row"], t["dl"],
                                         t.get("dz"), t["dWg"], t.get("dwsg"), ws)),
         ("unpermute_grad", lambda: B.unpermute_grad(c, t["dXp"], t["row_of_slot"], t.get("dXs"), t["idx"], t["dl"],
                                                     t["Wg"], t.get("dz"), t.get("wsg"), t["dX"])),
@@ -257,13 +265,15 @@ def dedup_dispatch_timing(lay, reps=5):
     Xr = torch.empty((cap, c.d), dtype=t["X"].dtype, device=dev)
     ws = torch.empty(B.workspace_bytes(c, B.WS_DISPATCH_DEDUP), dtype=torch.uint8, device=dev)
 
+    Xp = t["Xp"] if "Xp" in t else torch.empty((lay.R, c.d), dtype=t["X"].dtype, device=dev)
+
     def run_dedup():
         B.dispatch_dedup(c, t["idx"], t["part"], t.get("expert_rank"), t["X"], t["counts"], t["offsets"], t["row_of_slot"],
-                         t["slot_of_row"], rc, ro, rrs, tok, Xr, t["Xp"], t["status"], ws)
+                         t["slot_of_row"], rc, ro, rrs, tok, Xr, Xp, t["status"], ws)
 
     def run_plain():
         B.permute(c, t["idx"], t.get("expert_rank"), t["X"], t["counts"], t["offsets"], t["row_of_slot"], t["slot_of_row"],
-                  t["Xp"], t["status"], t["ws"])
+                  Xp, t["status"], t["ws"])
 
     res = {}
     for name, fn in (("dedup_two_stage", run_dedup), ("plain", run_plain)):
@@ -387,6 +397,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
     ap.add_argument("--no-reports", action="store_true", help="skip the Top-K vs C2R dispatch reports")
+    ap.add_argument("--dispatch", default="permute", choices=["permute", "gather-fused"],
+                    help="permute: c2r_permute writes Xp (faster); gather-fused: the expert GEMMs read token rows from X, no permuted copy")
     args = ap.parse_args()
 
     from paper_2504_01337_b200 import inputs as G
@@ -408,7 +420,8 @@ def main():
 
     # every rank is an independent data-parallel replica: same parameters, its own batch
     wl_rank = RP.rank_workload(wl, rank)
-    lay, cal = build_layer(wl, device, keep=True)
+    fused = args.dispatch == "gather-fused" and wl.bf16
+    lay, cal = build_layer(wl, device, keep=True, gather_fused=fused)
     if args.workload == "c5":
         # large-batch training step: the sets refreshed from this step's routing (Eq. 2, Eq. 4) are the
         # ones the next step routes with (the refresh is the last thing a step enqueues)
@@ -512,7 +525,7 @@ def main():
             "vs_baseline": None, "dtype": "bf16" if wl.bf16 else "f32", "data": "synthetic",
             "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "E": wl.E, "I": wl.I, "K": wl.K, "T": wl.T,
                        "P": wl.P, "I_s": wl.I_s, "row_align": lay.cfg.row_align, "parallelism": f"dp{world} (replicas)",
-                       "step": "fwd+bwd+collab refresh (c2r_train_step)",
+                       "step": "fwd+bwd+collab refresh (c2r_train_step)", "dispatch": "gather-fused" if fused else "permute",
                        "l2": "working set (>1 GB weights + activations) exceeds the 126 MB L2"},
             "clocks": clocks,
             "e2e": {"value": RP.whole_job_rate(wl.N, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": 2 * nbytes,
@@ -539,11 +552,11 @@ def main():
                                "flops_per_launch": fl_step / n_launch}
             es = 2 if wl.bf16 else 4
             sh = 1 if wl.I_s else 0
-            hb = {"permute": wl.N * wl.d * es * (wl.K + 1),
+            hb = {"permute": 0 if fused else wl.N * wl.d * es * (wl.K + 1),
                   "combine": wl.N * wl.d * (4 * wl.K + 4 * sh + es),
                   "combine_bwd": wl.N * wl.d * (4 * wl.K + 4 * sh + es + es * wl.K + es * sh),
                   "unpermute_grad": wl.N * wl.d * (4 * wl.K + 4 * sh + es)}
-            out["hbm_gbs"] = {k: hb[k] / (bd[k] * 1e-3) / 1e9 for k in hb}
+            out["hbm_gbs"] = {k: hb[k] / (bd[k] * 1e-3) / 1e9 for k in hb if hb[k]}
             out["hbm_frac_of_measured"] = {k: v / peaks["hbm_gbs"] for k, v in out["hbm_gbs"].items()}
         if not args.no_reports:
             out["dispatch_report"] = dispatch_report(lay.t["L"], lay.t["mask"] if args.workload != "c5" else mask_cal,

@@ -61,8 +61,14 @@ typedef struct c2r_config {
   int32_t row_align; /* every expert's segment of the permuted layout starts at a multiple of this
                         (>= 1; the tensor-core GEMMs of the bf16 path need a multiple of 128) */
   int32_t renorm;    /* 1: weights = softmax over the K kept logits (Eq. 1); 0: full-softmax probabilities */
-  int32_t flags;     /* reserved, 0 */
+  int32_t flags;     /* OR of C2R_FLAG_* */
 } c2r_config;
+
+/* c2r_config.flags */
+enum {
+  C2R_FLAG_GATHER_FUSED = 1 /* layer drivers (bf16 tensor-core path): the expert GEMMs fetch token rows straight
+                               from X through slot_of_row (TMA row gather); Xp is neither written nor read */
+};
 
 enum { C2R_WS_PERMUTE = 0, C2R_WS_GATE_BWD = 1, C2R_WS_LAYER = 2, C2R_WS_DISPATCH_DEDUP = 3 };
 
@@ -211,6 +217,22 @@ int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t 
                            const int32_t* counts, const int32_t* offsets, const void* W13p,
                            const void* W2, const void* AB, const void* H, const void* dYp, void* dAB,
                            void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status, void* stream);
+
+/* The two calls above with the dispatch folded into the GEMMs (an addition of this library: the gather-fused
+ * form of the dispatch): wherever they read row r of Xp, the kernels read row slot_of_row[r] / K of X
+ * instead (zeros where slot_of_row[r] < 0), so c2r_permute can be called with X == NULL and no permuted copy
+ * of the hidden states exists.  Same outputs, bit for bit.  bf16 tensor-core shapes only (d % 16 == 0,
+ * I % 16 == 0, row_align a multiple of 128): anything else returns C2R_ERR_UNSUPPORTED_SHAPE.
+ * X [N,d] T; slot_of_row [R] int32 as c2r_permute wrote it. */
+int c2r_grouped_swiglu_fwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
+                                  const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
+                                  const void* W13p, const void* W2, void* AB, void* H, void* Yp, int32_t* status,
+                                  void* stream);
+int c2r_grouped_swiglu_bwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
+                                  const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
+                                  const void* W13p, const void* W2, const void* AB, const void* H, const void* dYp,
+                                  void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status,
+                                  void* stream);
 
 /* Sec. 3.1 (weighted sum of the selected experts' outputs):
  * Y[t,:] = sum_k w[t,k] * Yp[row_of_slot[t*K+k],:]  (k ascending, fp32)

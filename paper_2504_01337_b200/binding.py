@@ -57,6 +57,7 @@ EXPORTS = [
     "c2r_unpack_weights", "c2r_grouped_swiglu_fwd", "c2r_grouped_swiglu_bwd", "c2r_combine", "c2r_combine_bwd",
     "c2r_route_bwd", "c2r_gate_bwd", "c2r_unpermute_grad", "c2r_dispatch_volume", "c2r_layer_fwd",
     "c2r_layer_bwd", "c2r_train_step", "c2r_permute_static", "c2r_dispatch_dedup",
+    "c2r_grouped_swiglu_fwd_gather", "c2r_grouped_swiglu_bwd_gather",
 ]
 
 _P = C.c_void_p
@@ -81,6 +82,8 @@ _SIGS = {
     "c2r_unpack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
     "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 10,
     "c2r_grouped_swiglu_bwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 12 + [C.c_int, _P, _P],
+    "c2r_grouped_swiglu_fwd_gather": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 11,
+    "c2r_grouped_swiglu_bwd_gather": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 13 + [C.c_int, _P, _P],
     "c2r_combine": [_CFG] + [_P] * 7,
     "c2r_combine_bwd": [_CFG] + [_P] * 12,
     "c2r_route_bwd": [_CFG] + [_P] * 4,
@@ -96,8 +99,11 @@ for _name, _sig in _SIGS.items():
     getattr(lib, _name).argtypes = _sig
 
 
-def make_config(N, d, E, I, K, T=0, P=1, I_s=0, dtype=BF16, row_align=1, renorm=1) -> Config:
-    return Config(N, d, E, I, K, T, P, I_s, dtype, row_align, renorm, 0)
+FLAG_GATHER_FUSED = 1
+
+
+def make_config(N, d, E, I, K, T=0, P=1, I_s=0, dtype=BF16, row_align=1, renorm=1, flags=0) -> Config:
+    return Config(N, d, E, I, K, T, P, I_s, dtype, row_align, renorm, flags)
 
 
 def _ptr(t):
@@ -200,6 +206,18 @@ def grouped_swiglu_bwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, 
                        accumulate=False, status=None):
     _call("c2r_grouped_swiglu_bwd", C.byref(cfg), n_experts, I, int(R), _ptr(Xp), _ptr(counts), _ptr(offsets),
           _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2),
+          int(accumulate), _ptr(status), _stream())
+
+
+def grouped_swiglu_fwd_gather(cfg, n_experts, I, R, X, slot_of_row, counts, offsets, W13p, W2, AB, H, Yp, status=None):
+    _call("c2r_grouped_swiglu_fwd_gather", C.byref(cfg), n_experts, I, int(R), _ptr(X), _ptr(slot_of_row), _ptr(counts),
+          _ptr(offsets), _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(Yp), _ptr(status), _stream())
+
+
+def grouped_swiglu_bwd_gather(cfg, n_experts, I, R, X, slot_of_row, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p,
+                              dW2, accumulate=False, status=None):
+    _call("c2r_grouped_swiglu_bwd_gather", C.byref(cfg), n_experts, I, int(R), _ptr(X), _ptr(slot_of_row), _ptr(counts),
+          _ptr(offsets), _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2),
           int(accumulate), _ptr(status), _stream())
 
 

@@ -106,6 +106,33 @@ extern "C" int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int 
                                         dW13p, dW2, accumulate, s);
 }
 
+extern "C" int c2r_grouped_swiglu_fwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
+                                             const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
+                                             const void* W13p, const void* W2, void* AB, void* H, void* Yp,
+                                             int32_t* status, void* stream) {
+  int rc = check_gemm_args(cfg, n_experts, I, R);
+  if (rc) return rc;
+  C2R_REQUIRE(X && slot_of_row && counts && offsets && W13p && W2 && H && Yp, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(tc_supported(cfg, n_experts, I, R) && (((uintptr_t)X) & 15u) == 0, C2R_ERR_UNSUPPORTED_SHAPE);
+  if (R == 0) return C2R_OK;
+  return tc_swiglu_fwd(cfg, n_experts, I, R, nullptr, counts, offsets, W13p, W2, AB, H, Yp, status, as_stream(stream), X,
+                       slot_of_row);
+}
+
+extern "C" int c2r_grouped_swiglu_bwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
+                                             const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
+                                             const void* W13p, const void* W2, const void* AB, const void* H,
+                                             const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2,
+                                             int accumulate, int32_t* status, void* stream) {
+  int rc = check_gemm_args(cfg, n_experts, I, R);
+  if (rc) return rc;
+  C2R_REQUIRE(X && slot_of_row && counts && offsets && W13p && W2 && AB && H && dYp && dAB && dXp && dW13p && dW2,
+              C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(tc_supported(cfg, n_experts, I, R) && (((uintptr_t)X) & 15u) == 0, C2R_ERR_UNSUPPORTED_SHAPE);
+  return tc_swiglu_bwd(cfg, n_experts, I, R, nullptr, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p, dW2, accumulate,
+                       status, as_stream(stream), X, slot_of_row);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Whole-layer drivers: the calls above chained on one stream, no host synchronisation.
 // ---------------------------------------------------------------------------------------------
@@ -114,6 +141,12 @@ extern "C" int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int 
     int _rc = (expr);         \
     if (_rc) return _rc;      \
   } while (0)
+
+// The gather-fused dispatch is used when asked for and the routed experts run on the tensor-core path.
+static bool gather_fused(const c2r_config* cfg, const void* X) {
+  return (cfg->flags & C2R_FLAG_GATHER_FUSED) != 0 && X != nullptr && (((uintptr_t)X) & 15u) == 0 &&
+         cfg->E < 64 && tc_supported(cfg, cfg->E, cfg->I, permuted_rows(cfg));
+}
 
 extern "C" int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, void* stream) {
   int rc = check_config(cfg);
@@ -127,10 +160,15 @@ extern "C" int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
   const int64_t R = permuted_rows(cfg);
   C2R_TRY(gate_logits_impl(cfg, b->X, b->Wg, shared ? b->wsg : nullptr, b->L, b->z, b->status, stream));
   C2R_TRY(c2r_route(cfg, b->L, b->mask, b->idx, b->w, nullptr, b->status, stream));
-  C2R_TRY(c2r_permute(cfg, b->idx, b->expert_rank, b->X, b->counts, b->offsets, b->row_of_slot, b->slot_of_row, b->Xp,
-                      b->status, b->ws, b->ws_bytes, stream));
-  C2R_TRY(c2r_grouped_swiglu_fwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
-                                 b->Yp, b->status, stream));
+  const bool fused = gather_fused(cfg, b->X);
+  C2R_TRY(c2r_permute(cfg, b->idx, b->expert_rank, fused ? nullptr : b->X, b->counts, b->offsets, b->row_of_slot,
+                      b->slot_of_row, b->Xp, b->status, b->ws, b->ws_bytes, stream));
+  if (fused)
+    C2R_TRY(c2r_grouped_swiglu_fwd_gather(cfg, cfg->E, cfg->I, R, b->X, b->slot_of_row, b->counts, b->offsets, b->W13p,
+                                          b->W2, b->AB, b->H, b->Yp, b->status, stream));
+  else
+    C2R_TRY(c2r_grouped_swiglu_fwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
+                                   b->Yp, b->status, stream));
   if (shared)
     C2R_TRY(c2r_grouped_swiglu_fwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
                                    b->Hs, b->Ys, b->status, stream));
@@ -158,8 +196,13 @@ extern "C" int c2r_layer_bwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
   C2R_TRY(c2r_combine_bwd(cfg, b->dY, b->Yp, b->w, b->row_of_slot, b->slot_of_row, shared ? b->Ys : nullptr,
                           shared ? b->z : nullptr, b->dYp, b->dw, shared ? b->dYs : nullptr,
                           shared ? b->dz : nullptr, stream));
-  C2R_TRY(c2r_grouped_swiglu_bwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
-                                 b->dYp, b->dAB, b->dXp, b->dW13p, b->dW2, accumulate, b->status, stream));
+  if (gather_fused(cfg, b->X))
+    C2R_TRY(c2r_grouped_swiglu_bwd_gather(cfg, cfg->E, cfg->I, R, b->X, b->slot_of_row, b->counts, b->offsets, b->W13p,
+                                          b->W2, b->AB, b->H, b->dYp, b->dAB, b->dXp, b->dW13p, b->dW2, accumulate,
+                                          b->status, stream));
+  else
+    C2R_TRY(c2r_grouped_swiglu_bwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
+                                   b->dYp, b->dAB, b->dXp, b->dW13p, b->dW2, accumulate, b->status, stream));
   if (shared)
     C2R_TRY(c2r_grouped_swiglu_bwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
                                    b->Hs, b->dYs, b->dABs, b->dXs, b->dWs13p, b->dWs2, accumulate, b->status, stream));

@@ -41,13 +41,15 @@ int simt_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void*
 enum { TC_ROWS = 0, TC_WGRAD = 1 };
 enum { TC_EPI_SWIGLU_FWD = 0, TC_EPI_F32 = 1, TC_EPI_SWIGLU_BWD = 2, TC_EPI_WGRAD_BF16 = 3, TC_EPI_T_F32 = 4 };
 bool tc_supported(const c2r_config* cfg, int nE, int I, int64_t R);
+// X / slot_of_row (both or neither): the rows of the permuted operand are fetched from X inside the kernels
+// (TMA row gather) and Xp is not read.
 int tc_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
                   const int32_t* offsets, const void* W13p, const void* W2, void* AB, void* H, void* Yp,
-                  int32_t* status, cudaStream_t s);
+                  int32_t* status, cudaStream_t s, const void* X = nullptr, const int32_t* slot_of_row = nullptr);
 int tc_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
                   const int32_t* offsets, const void* W13p, const void* W2, const void* AB, const void* H,
                   const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status,
-                  cudaStream_t s);
+                  cudaStream_t s, const void* X = nullptr, const int32_t* slot_of_row = nullptr);
 
 // Gate logits on the tensor cores (bf16 only).
 bool gate_tc_supported(const c2r_config* cfg);

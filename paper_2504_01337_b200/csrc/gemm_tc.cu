@@ -52,6 +52,10 @@ struct TcParams {
   const void* AB;  // TC_EPI_SWIGLU_BWD: saved (A, B)
   void* H;         // TC_EPI_SWIGLU_FWD: H output
   int32_t* status;
+  // row-gathering variants: the operand's rows are token rows of X picked through slot_of_row
+  const int32_t* slot_of_row;  // [R], -1 = padding (reads zeros)
+  int slots_per_token;         // K of the routing
+  int n_tokens;                // rows of X
 };
 
 struct TileInfo {
@@ -181,8 +185,20 @@ __device__ __forceinline__ void stage_rows_store(uint32_t buf, const uint4 (&v)[
   for (int it = 0; it < 8; ++it) sts128(stg_addr(buf, 4 * it + sub, chunk), v[it]);
 }
 
+// Token rows behind four consecutive rows r..r+3 of the permuted layout (r a multiple of 4): slot / K, and an
+// out-of-range row (-> zero fill) for padding or rows past the layout.
+__device__ __forceinline__ int4 gather_rows(const TcParams& p, int r) {
+  int4 s = make_int4(-1, -1, -1, -1);
+  if (r >= 0 && r + 3 < p.R) s = *reinterpret_cast<const int4*>(p.slot_of_row + r);
+  const int K = p.slots_per_token, oob = p.n_tokens;
+  return make_int4(s.x < 0 ? oob : s.x / K, s.y < 0 ? oob : s.y / K, s.z < 0 ? oob : s.z / K, s.w < 0 ? oob : s.w / K);
+}
+
 // A_MN / B_MN: operand is MN-major in global memory (the contraction index is the row index).
-template <bool A_MN, bool B_MN>
+// GATHER: 0 = both operands are plain arrays; 1 = A's rows (TC_ROWS, K-major) are token rows gathered from X;
+// 2 = B's contraction rows (TC_WGRAD, MN-major) are token rows gathered from X.  map_a / map_b is then the
+// one-row-box map of X, and the permuted copy of X is never needed.
+template <bool A_MN, bool B_MN, int GATHER>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -234,7 +250,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (warp == 0) {
     // ------------------------------- TMA producer (each CTA loads its own halves) ----------
-    if (lane == 0) {
+    // Lane 0 waits and issues the tiled loads; a gathered operand is fetched by all 32 lanes, four rows each.
+    {
       const uint32_t full_mma0 = map_to_cta(full0, 0);  // completion bytes are counted where the MMAs are issued
       uint32_t stage = 0, phase = 0;
       bool ok = true;
@@ -245,33 +262,51 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         n_geometry(p, ti.jn, n_mma, w, brow0);
         const int a0 = ti.m0 + BM * (int)rank;               // this CTA's A rows (or output-row range for MN-major A)
         const int b0 = brow0 + (n_mma >> 1) * (int)rank;     // this CTA's B rows
+        int4 rows = make_int4(0, 0, 0, 0);
+        if (GATHER == 1) rows = gather_rows(p, a0 + 4 * lane);                       // the same rows for every k-block
+        if (GATHER == 2) rows = gather_rows(p, ti.krow0 + 4 * (lane & 15));          // k-block 0; refreshed below
         for (int kb = 0; kb < ti.kblocks; ++kb) {
-          if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-          if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * STAGE_BYTES);
+          int4 next_rows = rows;
+          if (GATHER == 2 && kb + 1 < ti.kblocks) next_rows = gather_rows(p, ti.krow0 + (kb + 1) * BK + 4 * (lane & 15));
+          if (lane == 0) ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag);
+          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+          if (!ok) break;
+          if (lane == 0 && rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * STAGE_BYTES);
           const uint32_t fb = full_mma0 + 8 * stage;
           const uint32_t sa = smem_base + stage * STAGE_BYTES;
           const uint32_t sb = sa + HALF_BYTES;
-          if (!A_MN) {
-            tma_pair_load_2d(sa, &map_a, fb, kb * BK, a0);  // [128 rows][64 k]
-          } else {
-            const int kr = ti.krow0 + kb * BK;
-            tma_pair_load_2d(sa, &map_a, fb, a0, kr);  // [64 k][64 m] twice
-            tma_pair_load_2d(sa + 8192, &map_a, fb, a0 + 64, kr);
+          if (GATHER == 1) {
+            tma_pair_gather4(sa + 512 * lane, &map_a, fb, kb * BK, rows.x, rows.y, rows.z, rows.w);  // [128 rows][64 k]
+          } else if (lane == 0) {
+            if (!A_MN) {
+              tma_pair_load_2d(sa, &map_a, fb, kb * BK, a0);  // [128 rows][64 k]
+            } else {
+              const int kr = ti.krow0 + kb * BK;
+              tma_pair_load_2d(sa, &map_a, fb, a0, kr);  // [64 k][64 m] twice
+              tma_pair_load_2d(sa + 8192, &map_a, fb, a0 + 64, kr);
+            }
           }
-          if (!B_MN) {
-            tma_pair_load_3d(sb, &map_b, fb, kb * BK, b0, ti.expert);  // [128 n][64 k] of the expert's weights
-          } else if (p.mode == TC_ROWS) {
-            tma_pair_load_3d(sb, &map_b, fb, b0, kb * BK, ti.expert);  // [64 k][64 n] twice
-            tma_pair_load_3d(sb + 8192, &map_b, fb, b0 + 64, kb * BK, ti.expert);
-          } else {
-            const int kr = ti.krow0 + kb * BK;
-            tma_pair_load_2d(sb, &map_b, fb, b0, kr);
-            tma_pair_load_2d(sb + 8192, &map_b, fb, b0 + 64, kr);
+          if (GATHER == 2) {
+            // [64 k][64 n] twice: lanes 0..15 fill the first box, lanes 16..31 the second (64 columns further)
+            const int h = lane >> 4;
+            tma_pair_gather4(sb + 8192 * h + 512 * (lane & 15), &map_b, fb, b0 + 64 * h, rows.x, rows.y, rows.z, rows.w);
+          } else if (lane == 0) {
+            if (!B_MN) {
+              tma_pair_load_3d(sb, &map_b, fb, kb * BK, b0, ti.expert);  // [128 n][64 k] of the expert's weights
+            } else if (p.mode == TC_ROWS) {
+              tma_pair_load_3d(sb, &map_b, fb, b0, kb * BK, ti.expert);  // [64 k][64 n] twice
+              tma_pair_load_3d(sb + 8192, &map_b, fb, b0 + 64, kb * BK, ti.expert);
+            } else {
+              const int kr = ti.krow0 + kb * BK;
+              tma_pair_load_2d(sb, &map_b, fb, b0, kr);
+              tma_pair_load_2d(sb + 8192, &map_b, fb, b0 + 64, kr);
+            }
           }
+          rows = next_rows;
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) { *abort_flag = 1; if (p.status) atomicOr(p.status, C2R_STATUS_WAIT_TIMEOUT); }
+      if (!ok && lane == 0) { *abort_flag = 1; if (p.status) atomicOr(p.status, C2R_STATUS_WAIT_TIMEOUT); }
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer (even CTA of the pair) ----------------------
@@ -542,7 +577,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-template <bool A_MN, bool B_MN>
+template <bool A_MN, bool B_MN, int GATHER = 0>
 static int launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, cudaStream_t s) {
   constexpr int smem = SMEM_BYTES;
   constexpr int MAX_DEV = 64;
@@ -563,17 +598,17 @@ static int launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& 
   cfg.numAttrs = 1;
   int grid = __atomic_load_n(&grid_of_device[dev], __ATOMIC_ACQUIRE);
   if (grid == 0) {
-    C2R_CUDA(cudaFuncSetAttribute(tc_gemm_kernel<A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    C2R_CUDA(cudaFuncSetAttribute(tc_gemm_kernel<A_MN, B_MN, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     int sms = 0, pairs = 0;
     C2R_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     cfg.gridDim = dim3(sms / 2 * 2);
-    C2R_CUDA(cudaOccupancyMaxActiveClusters(&pairs, tc_gemm_kernel<A_MN, B_MN>, &cfg));
+    C2R_CUDA(cudaOccupancyMaxActiveClusters(&pairs, tc_gemm_kernel<A_MN, B_MN, GATHER>, &cfg));
     if (pairs < 1) return C2R_ERR_UNSUPPORTED_SHAPE;
     grid = 2 * (pairs < sms / 2 ? pairs : sms / 2);
     __atomic_store_n(&grid_of_device[dev], grid, __ATOMIC_RELEASE);
   }
   cfg.gridDim = dim3(grid);
-  C2R_CUDA(cudaLaunchKernelEx(&cfg, tc_gemm_kernel<A_MN, B_MN>, ma, mb, p));
+  C2R_CUDA(cudaLaunchKernelEx(&cfg, tc_gemm_kernel<A_MN, B_MN, GATHER>, ma, mb, p));
   C2R_LAUNCH_CHECK();
   return C2R_OK;
 }
@@ -587,18 +622,20 @@ bool tc_supported(const c2r_config* cfg, int nE, int I, int64_t R) {
 
 int tc_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
                   const int32_t* offsets, const void* W13p, const void* W2, void* AB, void* H, void* Yp,
-                  int32_t* status, cudaStream_t s) {
+                  int32_t* status, cudaStream_t s, const void* X, const int32_t* slot_of_row) {
   const int d = cfg->d;
   CUtensorMap ma, mb;
   TcParams p{};
   p.mode = TC_ROWS; p.n_experts = nE; p.R = (int)R; p.I = I; p.counts = counts; p.offsets = offsets; p.status = status;
   // (A | B) = Xp W13p^T with the SwiGLU epilogue: AB packed + H
-  int rc = make_map(&ma, Xp, d, R, 0, BK, BM);
+  const bool gather = X != nullptr && slot_of_row != nullptr;  // rows of X picked inside the GEMM, no permuted copy
+  int rc = gather ? make_map(&ma, X, d, cfg->N, 0, BK, 1) : make_map(&ma, Xp, d, R, 0, BK, BM);
   if (rc) return rc;
   rc = make_map(&mb, W13p, d, 2 * I, nE, BK, 128);
   if (rc) return rc;
   p.epi = TC_EPI_SWIGLU_FWD; p.K = d; p.Nout = I; p.n_tiles = (I + 127) / 128; p.C = AB; p.H = H;
-  rc = launch<false, false>(ma, mb, p, s);
+  p.slot_of_row = slot_of_row; p.slots_per_token = cfg->K; p.n_tokens = cfg->N;
+  rc = gather ? launch<false, false, 1>(ma, mb, p, s) : launch<false, false>(ma, mb, p, s);
   if (rc) return rc;
   // Yp = H W2^T (fp32)
   rc = make_map(&ma, H, I, R, 0, BK, BM);
@@ -612,7 +649,7 @@ int tc_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* X
 int tc_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
                   const int32_t* offsets, const void* W13p, const void* W2, const void* AB, const void* H,
                   const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status,
-                  cudaStream_t s) {
+                  cudaStream_t s, const void* X, const int32_t* slot_of_row) {
   const int d = cfg->d;
   CUtensorMap ma, mb;
   TcParams p{};
@@ -647,11 +684,13 @@ int tc_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* X
   // dW13p_e = dAB_e^T Xp_e  [2I, d]
   rc = make_map(&ma, dAB, 2 * I, R, 0, 64, 64);
   if (rc) return rc;
-  rc = make_map(&mb, Xp, d, R, 0, 64, 64);
+  const bool gather = X != nullptr && slot_of_row != nullptr;
+  rc = gather ? make_map(&mb, X, d, cfg->N, 0, 64, 1) : make_map(&mb, Xp, d, R, 0, 64, 64);
   if (rc) return rc;
   p.Mout = 2 * I; p.Nout = d; p.m_tiles = (2 * I + TILE_M - 1) / TILE_M; p.n_tiles = (d + TILE_N - 1) / TILE_N;
   p.C = dW13p; p.ldc = d; p.sC = (long long)2 * I * d;
-  return launch<true, true>(ma, mb, p, s);
+  p.slot_of_row = slot_of_row; p.slots_per_token = cfg->K; p.n_tokens = cfg->N;
+  return gather ? launch<true, true, 2>(ma, mb, p, s) : launch<true, true>(ma, mb, p, s);
 }
 
 int tc_gate_wgrad(const c2r_config* cfg, const void* X, const void* dLd, float* partial, int n_splits,

@@ -782,6 +782,7 @@ static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp,
     C2R_LAUNCH_CHECK();
     return C2R_OK;
   }
+  C2R_REQUIRE(Xp != nullptr, C2R_ERR_INVALID_ARG);  // the row-serial form walks the permuted rows
   const int colblocks = (cfg->d + 32 * V::N - 1) / (32 * V::N);
   gate_wgrad_kernel<T><<<dim3(colblocks, cfg->E), 256, 0, s>>>((const T*)Xp, counts, offsets, slot_of_row, dl, dWg,
                                                                cfg->d);
@@ -800,7 +801,7 @@ extern "C" int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp
                             float* dWg, float* dwsg, void* ws, size_t ws_bytes, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
-  C2R_REQUIRE(Xp && counts && offsets && slot_of_row && dl && dWg, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(counts && offsets && slot_of_row && dl && dWg, C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(!dz || (X && dwsg), C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(!dz || (ws && ws_bytes >= gate_bwd_ws_bytes(cfg)), C2R_ERR_WORKSPACE);
   if (ws && ws_bytes < gate_bwd_ws_bytes(cfg)) ws = nullptr;  // too small for the tensor-core form: row-serial kernel

@@ -130,6 +130,17 @@ __device__ __forceinline__ void tma_pair_load_3d(uint32_t dst, const CUtensorMap
       "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
+// Row-gathering TMA load (tile::gather4): four rows r0..r3 of a 2-D tensor whose map has a one-row box,
+// `x` the first column; the rows land one after the other (box-width bytes each) at dst.  A row index
+// outside the tensor reads the fill value (zeros).
+__device__ __forceinline__ void tma_pair_gather4(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int r0, int r1,
+                                                 int r2, int r3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, "
+      "%5, %6, %7}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+      : "memory");
+}
 // Arrives (once) on the barrier at the same offset in both CTAs when the MMAs issued so far are done.
 __device__ __forceinline__ void tc_pair_commit(uint32_t bar) {
   asm volatile(

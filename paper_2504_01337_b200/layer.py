@@ -21,10 +21,11 @@ class C2RLayer:
     to torch tensors."""
 
     def __init__(self, N, d, E, I, K, T, P, I_s=0, bf16=True, row_align=None, backward=True, profile=False,
-                 renorm=1, device="cuda"):
+                 renorm=1, device="cuda", gather_fused=False):
         if row_align is None:
             row_align = 128 if bf16 else 1
-        self.cfg = B.make_config(N, d, E, I, K, T, P, I_s, B.BF16 if bf16 else B.F32, row_align, renorm)
+        self.cfg = B.make_config(N, d, E, I, K, T, P, I_s, B.BF16 if bf16 else B.F32, row_align, renorm,
+                                 B.FLAG_GATHER_FUSED if gather_fused else 0)
         self.bf16 = bf16
         self.device = device
         self.R = B.permuted_rows(self.cfg)
@@ -44,7 +45,8 @@ class C2RLayer:
         t["offsets"] = buf((E + 1,), i32)
         t["row_of_slot"] = buf((N * K,), i32)
         t["slot_of_row"] = buf((R,), i32)
-        t["Xp"] = buf((R, d))
+        if not (gather_fused and bf16):  # the gather-fused GEMMs read token rows from X: no permuted copy
+            t["Xp"] = buf((R, d))
         t["H"] = buf((R, I))
         t["Yp"] = buf((R, d), f32)
         t["Y"] = buf((N, d))

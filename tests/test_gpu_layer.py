@@ -291,3 +291,37 @@ def test_weight_gradients_accumulate():
         twice = lay.t[k].float()
         # 2x is exact in bf16 up to the rounding of the sum: within one bf16 ulp of 2v
         assert torch.all((twice - 2 * v).abs() <= 2.0 ** -7 * (2 * v).abs() + 1e-30), k
+
+
+@pytest.mark.parametrize("N,d,E,I,K,T,P,I_s", [(2048, 256, 8, 400, 4, 5, 4, 528), (1500, 128, 6, 272, 3, 4, 3, 0),
+                                               (70, 64, 4, 16, 2, 2, 2, 0), (4096, 2048, 60, 1408, 4, 16, 4, 0)])
+def test_gather_fused_dispatch_is_bit_identical(N, d, E, I, K, T, P, I_s):
+    """The gather-fused drivers (expert GEMMs fetch token rows from X through slot_of_row, no permuted copy)
+    against the plain ones: every output, intermediate and gradient identical bit for bit."""
+    wl = G.Workload("gf", N=N, d=d, E=E, I=I, K=K, T=T, P=P, I_s=I_s, bf16=True, seed=31)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    sh = G.shared_weights(wl) if I_s else None
+    sets = random_sets(E, T, seed=6)
+    rank = np.random.default_rng(5).permutation(E)
+    layers = []
+    for fused in (False, True):
+        lay = _layer(wl, backward=True, gather_fused=fused)
+        lay.set_params(Wg, W1, W3, W2, wsg, sh)
+        lay.set_routing(mask=mask_of(sets, E), expert_rank=rank)
+        lay.set_input(X, dY)
+        for name in ("AB", "H", "Yp", "dAB", "dXp", "dW13p", "dW2", "Y", "dX", "dWg"):
+            lay.t[name].fill_(7.0)  # nothing may survive from the allocation
+        lay.forward()
+        lay.backward()
+        torch.cuda.synchronize()
+        assert int(lay.t["status"].item()) == 0
+        layers.append(lay)
+    plain, fused = layers
+    assert "Xp" in plain.t and "Xp" not in fused.t
+    n_rows = int(plain.t["offsets"][E].item())
+    for name in ("idx", "counts", "offsets", "row_of_slot", "Y", "dX", "dW13p", "dW2", "dWg"):
+        assert torch.equal(plain.t[name], fused.t[name]), name
+    for name in ("H", "AB", "Yp", "dAB", "dXp"):  # rows of the layout (beyond its end nothing is written)
+        assert torch.equal(plain.t[name][:n_rows], fused.t[name][:n_rows]), name
