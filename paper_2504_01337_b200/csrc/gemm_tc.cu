@@ -250,34 +250,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (warp == 0) {
     // ------------------------------- TMA producer (each CTA loads its own halves) ----------
-    // Lane 0 waits and issues the tiled loads; a gathered operand is fetched by all 32 lanes, four rows each.
-    {
-      const uint32_t full_mma0 = map_to_cta(full0, 0);  // completion bytes are counted where the MMAs are issued
-      uint32_t stage = 0, phase = 0;
-      bool ok = true;
-      for (long long t = pair_id; ok; t += n_pairs) {
-        TileInfo ti;
-        if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti)) break;
-        int n_mma, w, brow0;
-        n_geometry(p, ti.jn, n_mma, w, brow0);
-        const int a0 = ti.m0 + BM * (int)rank;               // this CTA's A rows (or output-row range for MN-major A)
-        const int b0 = brow0 + (n_mma >> 1) * (int)rank;     // this CTA's B rows
-        int4 rows = make_int4(0, 0, 0, 0);
-        if (GATHER == 1) rows = gather_rows(p, a0 + 4 * lane);                       // the same rows for every k-block
-        if (GATHER == 2) rows = gather_rows(p, ti.krow0 + 4 * (lane & 15));          // k-block 0; refreshed below
-        for (int kb = 0; kb < ti.kblocks; ++kb) {
-          int4 next_rows = rows;
-          if (GATHER == 2 && kb + 1 < ti.kblocks) next_rows = gather_rows(p, ti.krow0 + (kb + 1) * BK + 4 * (lane & 15));
-          if (lane == 0) ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag);
-          ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
-          if (!ok) break;
-          if (lane == 0 && rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * STAGE_BYTES);
-          const uint32_t fb = full_mma0 + 8 * stage;
-          const uint32_t sa = smem_base + stage * STAGE_BYTES;
-          const uint32_t sb = sa + HALF_BYTES;
-          if (GATHER == 1) {
-            tma_pair_gather4(sa + 512 * lane, &map_a, fb, kb * BK, rows.x, rows.y, rows.z, rows.w);  // [128 rows][64 k]
-          } else if (lane == 0) {
+    if constexpr (GATHER == 0) {
+      // plain operands: one thread waits for a free stage and issues the 2 to 4 tiled loads of a k-block
+      if (lane == 0) {
+        const uint32_t full_mma0 = map_to_cta(full0, 0);  // completion bytes are counted where the MMAs are issued
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (long long t = pair_id; ok; t += n_pairs) {
+          TileInfo ti;
+          if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti)) break;
+          int n_mma, w, brow0;
+          n_geometry(p, ti.jn, n_mma, w, brow0);
+          const int a0 = ti.m0 + BM * (int)rank;               // this CTA's A rows (or output-row range for MN-major A)
+          const int b0 = brow0 + (n_mma >> 1) * (int)rank;     // this CTA's B rows
+          for (int kb = 0; kb < ti.kblocks; ++kb) {
+            if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+            if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * STAGE_BYTES);
+            const uint32_t fb = full_mma0 + 8 * stage;
+            const uint32_t sa = smem_base + stage * STAGE_BYTES;
+            const uint32_t sb = sa + HALF_BYTES;
             if (!A_MN) {
               tma_pair_load_2d(sa, &map_a, fb, kb * BK, a0);  // [128 rows][64 k]
             } else {
@@ -285,12 +276,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               tma_pair_load_2d(sa, &map_a, fb, a0, kr);  // [64 k][64 m] twice
               tma_pair_load_2d(sa + 8192, &map_a, fb, a0 + 64, kr);
             }
-          }
-          if (GATHER == 2) {
-            // [64 k][64 n] twice: lanes 0..15 fill the first box, lanes 16..31 the second (64 columns further)
-            const int h = lane >> 4;
-            tma_pair_gather4(sb + 8192 * h + 512 * (lane & 15), &map_b, fb, b0 + 64 * h, rows.x, rows.y, rows.z, rows.w);
-          } else if (lane == 0) {
             if (!B_MN) {
               tma_pair_load_3d(sb, &map_b, fb, kb * BK, b0, ti.expert);  // [128 n][64 k] of the expert's weights
             } else if (p.mode == TC_ROWS) {
@@ -301,12 +286,71 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               tma_pair_load_2d(sb, &map_b, fb, b0, kr);
               tma_pair_load_2d(sb + 8192, &map_b, fb, b0 + 64, kr);
             }
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
           }
-          rows = next_rows;
-          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
+        if (!ok) { *abort_flag = 1; if (p.status) atomicOr(p.status, C2R_STATUS_WAIT_TIMEOUT); }
       }
-      if (!ok && lane == 0) { *abort_flag = 1; if (p.status) atomicOr(p.status, C2R_STATUS_WAIT_TIMEOUT); }
+    } else {
+      // a gathered operand: lane 0 waits and issues the tiled loads of the other operand, all 32 lanes fetch four
+      // token rows each
+      {
+        const uint32_t full_mma0 = map_to_cta(full0, 0);  // completion bytes are counted where the MMAs are issued
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (long long t = pair_id; ok; t += n_pairs) {
+          TileInfo ti;
+          if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti)) break;
+          int n_mma, w, brow0;
+          n_geometry(p, ti.jn, n_mma, w, brow0);
+          const int a0 = ti.m0 + BM * (int)rank;               // this CTA's A rows (or output-row range for MN-major A)
+          const int b0 = brow0 + (n_mma >> 1) * (int)rank;     // this CTA's B rows
+          int4 rows = make_int4(0, 0, 0, 0);
+          if (GATHER == 1) rows = gather_rows(p, a0 + 4 * lane);                       // the same rows for every k-block
+          if (GATHER == 2) rows = gather_rows(p, ti.krow0 + 4 * (lane & 15));          // k-block 0; refreshed below
+          for (int kb = 0; kb < ti.kblocks; ++kb) {
+            int4 next_rows = rows;
+            if (GATHER == 2 && kb + 1 < ti.kblocks) next_rows = gather_rows(p, ti.krow0 + (kb + 1) * BK + 4 * (lane & 15));
+            if (lane == 0) ok = mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag);
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            if (!ok) break;
+            if (lane == 0 && rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * STAGE_BYTES);
+            const uint32_t fb = full_mma0 + 8 * stage;
+            const uint32_t sa = smem_base + stage * STAGE_BYTES;
+            const uint32_t sb = sa + HALF_BYTES;
+            if (GATHER == 1) {
+              tma_pair_gather4(sa + 512 * lane, &map_a, fb, kb * BK, rows.x, rows.y, rows.z, rows.w);  // [128 rows][64 k]
+            } else if (lane == 0) {
+              if (!A_MN) {
+                tma_pair_load_2d(sa, &map_a, fb, kb * BK, a0);  // [128 rows][64 k]
+              } else {
+                const int kr = ti.krow0 + kb * BK;
+                tma_pair_load_2d(sa, &map_a, fb, a0, kr);  // [64 k][64 m] twice
+                tma_pair_load_2d(sa + 8192, &map_a, fb, a0 + 64, kr);
+              }
+            }
+            if (GATHER == 2) {
+              // [64 k][64 n] twice: lanes 0..15 fill the first box, lanes 16..31 the second (64 columns further)
+              const int h = lane >> 4;
+              tma_pair_gather4(sb + 8192 * h + 512 * (lane & 15), &map_b, fb, b0 + 64 * h, rows.x, rows.y, rows.z, rows.w);
+            } else if (lane == 0) {
+              if (!B_MN) {
+                tma_pair_load_3d(sb, &map_b, fb, kb * BK, b0, ti.expert);  // [128 n][64 k] of the expert's weights
+              } else if (p.mode == TC_ROWS) {
+                tma_pair_load_3d(sb, &map_b, fb, b0, kb * BK, ti.expert);  // [64 k][64 n] twice
+                tma_pair_load_3d(sb + 8192, &map_b, fb, b0 + 64, kb * BK, ti.expert);
+              } else {
+                const int kr = ti.krow0 + kb * BK;
+                tma_pair_load_2d(sb, &map_b, fb, b0, kr);
+                tma_pair_load_2d(sb + 8192, &map_b, fb, b0 + 64, kr);
+              }
+            }
+            rows = next_rows;
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+          }
+        }
+        if (!ok && lane == 0) { *abort_flag = 1; if (p.status) atomicOr(p.status, C2R_STATUS_WAIT_TIMEOUT); }
+      }
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer (even CTA of the pair) ----------------------
