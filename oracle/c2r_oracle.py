@@ -10,8 +10,8 @@ paper is silent the reading taken is stated in the docstring.
 Pins (see tests/test_oracle_*.py): brute-force enumeration of routing choices, the T = E-1
 degenerate case of Fig. 3, the uniform-routing closed form for redundancy (which also
 reproduces the Top-K rows implied by Tables 1 and 3), the structural zero pattern of Fig. 2,
-Eq. 2's invariants, a triple-loop dense SwiGLU, and central finite differences for every
-backward formula.
+Eq. 2's invariants, a triple-loop dense SwiGLU, central finite differences for every
+backward formula, and hand-worked values for the Eq. 1 weights and the load-imbalance statistics.
 Parity unpinned: the NaN ordering policy in `_order_desc` and the quality (not the rule) of
 `place_experts` -- the paper defines neither.
 """

@@ -106,6 +106,33 @@ def test_route_invariants_and_weights():
     assert np.count_nonzero(C1 - np.diag(np.diag(C1))) == 0
 
 
+def test_route_weights_and_load_stats_hand_values():
+    """Values worked out by hand, not by the formulas under test."""
+    # Eq. 1 on two kept logits 0 and ln 3: e^0 : e^{ln 3} = 1 : 3  ->  weights 1/4, 3/4
+    L = np.array([[0.0, np.log(3.0), -5.0]])
+    w = O.route_weights(L, np.array([[0, 1]]))
+    assert np.allclose(w, [[0.25, 0.75]], atol=1e-15)
+    # selection order is the order of `idx`: swapping the kept experts swaps the weights
+    assert np.allclose(O.route_weights(L, np.array([[1, 0]])), [[0.75, 0.25]], atol=1e-15)
+    # three kept logits ln 1, ln 2, ln 5 -> 1/8, 2/8, 5/8, whatever the common shift
+    L3 = np.array([[np.log(1.0), np.log(2.0), np.log(5.0)]]) + 123.0
+    assert np.allclose(O.route_weights(L3, np.array([[0, 1, 2]])), [[0.125, 0.25, 0.625]], atol=1e-12)
+    # without renormalisation the kept experts keep their share of the full softmax: logits ln 1, ln 1, ln 2
+    # have probabilities 1/4, 1/4, 1/2; keeping experts 2 and 0 gives 1/2, 1/4
+    Lf = np.array([[0.0, 0.0, np.log(2.0)]])
+    assert np.allclose(O.route_weights(Lf, np.array([[2, 0]]), renorm=False), [[0.5, 0.25]], atol=1e-15)
+    # load imbalance of counts [1, 1, 2]: mean 4/3, max/mean = 2 / (4/3) = 1.5;
+    # population variance = ((1/3)^2 + (1/3)^2 + (2/3)^2) / 3 = 2/9, std = sqrt(2)/3, cv = sqrt(2)/4
+    s = O.load_stats([1, 1, 2])
+    assert abs(s["max_over_mean"] - 1.5) < 1e-15 and abs(s["cv"] - 2.0 ** 0.5 / 4.0) < 1e-15
+    # perfectly balanced load: 1 and 0; one expert takes everything out of four: max/mean 4, cv sqrt(3)
+    s = O.load_stats([7, 7, 7, 7])
+    assert s == {"max_over_mean": 1.0, "cv": 0.0}
+    s = O.load_stats([0, 12, 0, 0])
+    assert abs(s["max_over_mean"] - 4.0) < 1e-15 and abs(s["cv"] - 3.0 ** 0.5) < 1e-12
+    assert O.load_stats([0, 0]) == {"max_over_mean": 0.0, "cv": 0.0}
+
+
 def test_nan_and_inf_order_last():
     L = np.array([[np.nan, 1.0, -np.inf, 0.5], [-np.inf, -np.inf, np.nan, -np.inf]], dtype=np.float32)
     idx, _ = O.topk_route(L, 3)
