@@ -35,6 +35,31 @@ def flops_per_token(wl):
     return 3 * (6 * wl.K * wl.d * wl.I + 6 * wl.d * wl.I_s)
 
 
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def hbm_bytes(wl, gather_fused=False):
+    """Bytes per step of the bandwidth-bound calls, two ways.  `moved`: what the kernels read and write
+    (the per-(token, expert) partial results Yp / dXp / Ys / dXs are stored in fp32).  `algorithmic`: what
+    the method has to move with every tensor in its storage type (gate: X once + L; route: L + idx + w;
+    dispatch: X once + K copies; combine and gradient un-permute: K (+1 shared) rows in, one row out)."""
+    es = 2 if wl.bf16 else 4
+    sh = 1 if wl.I_s else 0
+    N, d, E, K = wl.N, wl.d, wl.E, wl.K
+    index = 4 * N * K * 4                       # idx in, row_of_slot / slot_of_row / w_row out
+    rows = 0 if gather_fused else N * d * es * (K + 1)
+    moved = {"gate_logits": N * d * es + (E + sh) * d * es + N * (E + sh) * 4,
+             "route": N * E * 4 + 2 * N * K * 4,
+             "permute": rows + index,
+             "combine": N * d * (4 * K + 4 * sh + es),
+             "spread_dY": N * d * es * (K + 1),
+             "unpermute_grad": N * d * (4 * K + 4 * sh + es)}
+    alg = dict(moved)
+    alg["combine"] = N * d * es * (K + sh + 1)
+    alg["unpermute_grad"] = N * d * es * (K + sh + 1)
+    return moved, alg
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -62,7 +87,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -147,8 +172,8 @@ def build_layer(wl, device, profile=True, keep=False, gather_fused=False):
 
 def breakdown(lay, reps=3):
     """Per-call device time (ms) of one step: the calls c2r_train_step chains, issued one by one on
-    the same stream with a CUDA event between them, `reps` steps back to back (a sustained loop,
-    so the GEMM figures see the same power-capped clocks as the timed region)."""
+    one stream with a CUDA event between them, `reps` steps back to back (a sustained loop, so the
+    GEMM figures see the same power-capped clocks as the timed region)."""
     import torch
     from paper_2504_01337_b200 import binding as B
     c, t = lay.cfg, lay.t
@@ -157,40 +182,51 @@ def breakdown(lay, reps=3):
     R = lay.R
     P = c.P
     ws = t["ws"]
+    nq = B.swiglu_qparts(c, c.E, c.I, R)
+    nqs = B.swiglu_qparts(c, 1, c.I_s, c.N) if shared else 0
+    qpart = torch.empty((max(nq, 1), R), dtype=torch.float32, device=t["X"].device)
+    qspart = torch.empty((max(nqs, 1), c.N), dtype=torch.float32, device=t["X"].device)
+    row = dict(row_scale=t["w_row"], scale_kind=B.SCALE_ROW)
+    gate = dict(row_scale=t.get("z"), scale_kind=B.SCALE_SIGMOID)
     calls = [
         ("gate_logits", lambda: B.gate_logits(c, t["X"], t["Wg"], t.get("wsg"), t["L"], t.get("z"))),
-        ("route", lambda: B.route(c, t["L"], t.get("mask"), t["idx"], t["w"], None, t["status"])),
+        ("route", lambda: B.route(c, t["L"], t.get("mask"), t["idx"], t["w"], None, t["status"], ws)),
         ("permute", lambda: B.permute(c, t["idx"], t.get("expert_rank"), None if fused else t["X"], t["counts"],
-                                      t["offsets"], t["row_of_slot"], t["slot_of_row"], t.get("Xp"), t["status"], ws)),
+                                      t["offsets"], t["row_of_slot"], t["slot_of_row"], t.get("Xp"), t["status"], ws,
+                                      t["w"], t["w_row"], True)),
         ("swiglu_fwd", (lambda: B.grouped_swiglu_fwd_gather(c, c.E, c.I, R, t["X"], t["slot_of_row"], t["counts"],
-                                                            t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["Yp"]))
+                                                            t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["Yp"],
+                                                            None, **row))
          if fused else
          (lambda: B.grouped_swiglu_fwd(c, c.E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"],
-                                       t["W2"], t["AB"], t["H"], t["Yp"]))),
+                                       t["W2"], t["AB"], t["H"], t["Yp"], None, **row))),
     ]
     if shared:
         calls.append(("shared_fwd", lambda: B.grouped_swiglu_fwd(c, 1, c.I_s, c.N, t["X"], t["s_counts"], t["s_offsets"],
-                                                                 t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["Ys"])))
+                                                                 t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["Ys"], None,
+                                                                 **gate)))
     calls += [
-        ("combine", lambda: B.combine(c, t["Yp"], t["w"], t["row_of_slot"], t.get("Ys"), t.get("z"), t["Y"])),
+        ("combine", lambda: B.combine(c, t["Yp"], None, t["row_of_slot"], t.get("Ys"), None, t["Y"])),
         ("dispatch_volume", lambda: B.dispatch_volume(c, t["idx"], t["part"], t["volume"], t["volume"][4:],
                                                       t["volume"][4 + P * P:])),
-        ("combine_bwd", lambda: B.combine_bwd(c, t["dY"], t["Yp"], t["w"], t["row_of_slot"], t["slot_of_row"],
-                                              t.get("Ys"), t.get("z"), t["dYp"], t["dw"], t.get("dYs"), t.get("dz"))),
+        ("spread_dY", lambda: B.permute_rows(c, t["dY"], t["row_of_slot"], t["counts"], t["offsets"], t["dYp"])),
         ("swiglu_bwd", (lambda: B.grouped_swiglu_bwd_gather(c, c.E, c.I, R, t["X"], t["slot_of_row"], t["counts"],
                                                             t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["dYp"],
-                                                            t["dAB"], t["dXp"], t["dW13p"], t["dW2"]))
+                                                            t["dAB"], t["dXp"], t["dW13p"], t["dW2"], False, None,
+                                                            qpart=qpart, **row))
          if fused else
          (lambda: B.grouped_swiglu_bwd(c, c.E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"],
                                        t["W2"], t["AB"], t["H"], t["dYp"], t["dAB"], t["dXp"],
-                                       t["dW13p"], t["dW2"]))),
+                                       t["dW13p"], t["dW2"], False, None, qpart=qpart, **row))),
     ]
     if shared:
         calls.append(("shared_bwd", lambda: B.grouped_swiglu_bwd(c, 1, c.I_s, c.N, t["X"], t["s_counts"], t["s_offsets"],
-                                                                 t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["dYs"],
-                                                                 t["dABs"], t["dXs"], t["dWs13p"], t["dWs2"])))
+                                                                 t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["dY"],
+                                                                 t["dABs"], t["dXs"], t["dWs13p"], t["dWs2"], False, None,
+                                                                 qpart=qspart, **gate)))
     calls += [
-        ("route_bwd", lambda: B.route_bwd(c, t["w"], t["dw"], t["dl"])),
+        ("route_bwd", lambda: B.route_bwd_scaled(c, t["w"], t["row_of_slot"], qpart, nq, t.get("z"), qspart, nqs,
+                                                 t["dw"], t["dl"], t.get("dz"))),
         ("gate_bwd", lambda: B.gate_bwd(c, t["X"], t.get("Xp"), t["counts"], t["offsets"], t["slot_of_row"], t["dl"],
                                         t.get("dz"), t["dWg"], t.get("dwsg"), ws)),
         ("unpermute_grad", lambda: B.unpermute_grad(c, t["dXp"], t["row_of_slot"], t.get("dXs"), t["idx"], t["dl"],
@@ -367,7 +403,9 @@ def run_reference(args, wl):
         dt, state = cpu_oracle_step(wl, n_tok, state)
         total += dt
     val = n_tok * args.steps / total if total > 0 else 0.0
-    sample = f"first {n_tok} tokens of {wl.name} per step (all {wl.E} experts + shared expert), fwd+bwd, numpy fp64"
+    sample = (f"first {n_tok} tokens of {wl.name} per step (all {wl.E} experts + shared expert), fwd+bwd, numpy fp64; "
+              "the rate depends on the sample size: every expert's weights are touched whatever the token count, so "
+              "a larger sample amortises that fixed cost (the c2r arm's cpu_baseline uses a larger sample)")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * total / max(args.steps, 1), "higher_is_better": True,
@@ -550,14 +588,16 @@ def main():
                                "kernel": "tc_gemm_kernel (grouped SwiGLU GEMMs, routed + shared, fwd + bwd)",
                                "launches_per_step": n_launch, "avg_launch_ms": gemm_ms / n_launch,
                                "flops_per_launch": fl_step / n_launch}
-            es = 2 if wl.bf16 else 4
-            sh = 1 if wl.I_s else 0
-            hb = {"permute": 0 if fused else wl.N * wl.d * es * (wl.K + 1),
-                  "combine": wl.N * wl.d * (4 * wl.K + 4 * sh + es),
-                  "combine_bwd": wl.N * wl.d * (4 * wl.K + 4 * sh + es + es * wl.K + es * sh),
-                  "unpermute_grad": wl.N * wl.d * (4 * wl.K + 4 * sh + es)}
-            out["hbm_gbs"] = {k: hb[k] / (bd[k] * 1e-3) / 1e9 for k in hb if hb[k]}
+            out["roofline"].update({"frac_of_sustained": ach / peaks["bf16_tflops_sustained"],
+                                    "frac_of_burst": ach / peaks["bf16_tflops"],
+                                    "frac_of_nominal": ach / NOMINAL_BF16_TFLOPS,
+                                    "nominal_peak": NOMINAL_BF16_TFLOPS,
+                                    "nominal_source": "vendor dense bf16 figure for B200 (2.25 PFLOP/s; the doubled figure is 2:4 sparsity)"})
+            moved, alg = hbm_bytes(wl, fused)
+            out["hbm_gbs"] = {k: moved[k] / (bd[k] * 1e-3) / 1e9 for k in moved if moved[k]}
             out["hbm_frac_of_measured"] = {k: v / peaks["hbm_gbs"] for k, v in out["hbm_gbs"].items()}
+            out["hbm_gbs_algorithmic"] = {k: alg[k] / (bd[k] * 1e-3) / 1e9 for k in alg if alg[k]}
+            out["hbm_frac_of_measured_algorithmic"] = {k: v / peaks["hbm_gbs"] for k, v in out["hbm_gbs_algorithmic"].items()}
         if not args.no_reports:
             out["dispatch_report"] = dispatch_report(lay.t["L"], lay.t["mask"] if args.workload != "c5" else mask_cal,
                                                      cal["C"].cpu(), wl.E, wl.K, wl.T)
@@ -569,7 +609,9 @@ def main():
             dt, _ = cpu_oracle_step(wl, n_tok, st)
             out["cpu_baseline"] = {"value": n_tok / dt, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                                    "sample": f"one fwd+bwd step of the oracle on the first {n_tok} tokens of {wl.name} "
-                                             f"(all experts + shared expert), {dt:.1f} s"}
+                                             f"(all experts + shared expert), {dt:.1f} s; the rate depends on the sample "
+                                             "size (per-expert fixed cost), so --impl reference, which uses fewer "
+                                             "tokens per step, reports a lower one"}
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()

@@ -72,6 +72,11 @@ enum {
 
 enum { C2R_WS_PERMUTE = 0, C2R_WS_GATE_BWD = 1, C2R_WS_LAYER = 2, C2R_WS_DISPATCH_DEDUP = 3 };
 
+/* Per-row scale s_r the grouped SwiGLU calls can apply to H = s_r silu(A) B (and undo in their backward):
+ * none, s_r = row_scale[r] (the Eq. 1 weight of the row's slot), or s_r = sigmoid(row_scale[r]) (the
+ * shared expert's gate from its logit). */
+enum { C2R_SCALE_NONE = 0, C2R_SCALE_ROW = 1, C2R_SCALE_SIGMOID = 2 };
+
 /* Bytes of scratch the named call needs for this configuration (host function). */
 size_t c2r_workspace_bytes(const c2r_config* cfg, int which);
 
@@ -96,9 +101,12 @@ int c2r_gate_logits(const c2r_config* cfg, const void* X, const void* Wg, const 
  * NaN orders as -inf.  Selection is made on the raw fp32 logits.
  * L [N,E] float; mask [E] uint64 or NULL;
  * out: idx [N,K] int32 (column 0 = top-1, then selection order); w [N,K] float (Eq. 1 weights);
- *      p [N,E] float full-row softmax or NULL; status: one int32 (OR of C2R_STATUS_*) or NULL. */
+ *      p [N,E] float full-row softmax or NULL; status: one int32 (OR of C2R_STATUS_*) or NULL;
+ *      permute_ws (optional, C2R_WS_PERMUTE bytes): receives the per-block expert histogram of idx that
+ *      c2r_permute starts from; hand the same buffer to c2r_permute with ws_has_histogram = 1 and it skips
+ *      its own histogram pass. */
 int c2r_route(const c2r_config* cfg, const float* L, const uint64_t* mask, int32_t* idx, float* w,
-              float* p, int32_t* status, void* stream);
+              float* p, int32_t* status, void* permute_ws, void* stream);
 
 /* Sec. 3.2, Eq. 2: C[i,j] = number of tokens whose selected set contains both i and j.
  * idx [n_tokens,K] int32; C [E,E] int32.  accumulate != 0 adds to C (profiling over several
@@ -116,7 +124,7 @@ int c2r_collab_sets(const c2r_config* cfg, const int32_t* C, int32_t* I_T, uint6
  * C [E,E] int32; out: degree [E] float; mean (one float, may be NULL) = the layer's average over experts. */
 int c2r_collab_degree(const c2r_config* cfg, const int32_t* C, float* degree, float* mean, void* stream);
 
-/* Sec. 3.4 (co-locate closely collaborating experts on one device).  HOST function, host arrays.
+/* Sec. 3.4: placement of the experts on devices by collaboration.  HOST function, host arrays.
  * mode 0 (greedy): partition p holds floor(E/P) + (p < E mod P) experts; it is seeded with the
  * unassigned expert of largest C[e,e] and grown by the unassigned expert with the largest summed
  * co-activation with its members (ties: lower id).  mode 1: part[e] = floor(e*P/E).
@@ -131,11 +139,20 @@ int c2r_place_experts(const c2r_config* cfg, const int32_t* C_host, int mode, in
  * offsets[E] = end of the layout); row_of_slot [N*K] int32; slot_of_row [c2r_permuted_rows] int32
  * (-1 = padding); Xp [c2r_permuted_rows, d] T with Xp[r,:] = X[slot_of_row[r]/K,:]; the padding rows that
  * close an expert's aligned segment are zero, rows at or beyond offsets[E] are not written.
- * X == NULL builds the index only.  Atomic-free and deterministic.
- * ws: C2R_WS_PERMUTE bytes.  status as in c2r_route. */
-int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
-                int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp,
-                int32_t* status, void* ws, size_t ws_bytes, void* stream);
+ * X == NULL builds the index only.  w [N,K] float (optional) with w_row [c2r_permuted_rows] float (optional):
+ * w_row[r] = w[slot_of_row[r]], 0 on rows without a slot -- the per-row scale of the expert calls below.
+ * Atomic-free and deterministic.  An expert_rank that is not a permutation of [0,E) is replaced by the
+ * identity order and reported as C2R_STATUS_BAD_INDEX.  ws: C2R_WS_PERMUTE bytes; ws_has_histogram != 0: c2r_route
+ * already left the histogram of this very idx there.  status as in c2r_route. */
+int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X, const float* w,
+                int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp, float* w_row,
+                int32_t* status, void* ws, size_t ws_bytes, int ws_has_histogram, void* stream);
+
+/* The row gather of c2r_permute alone, for another [N,d] tensor and an index already built (the backward
+ * pass spreads dY this way: every permuted row receives its token's row unchanged).
+ * Xp[row_of_slot[t*K+k],:] = X[t,:]; padding rows that close an aligned segment are zeroed. */
+int c2r_permute_rows(const c2r_config* cfg, const void* X, const int32_t* row_of_slot, const int32_t* counts,
+                     const int32_t* offsets, void* Xp, void* stream);
 
 /* Sec. 3.4 (zero-redundancy all-to-all), carried out on one device in its two stages.
  * Stage 1: every token is copied ONCE to each partition that hosts at least one of its selected
@@ -167,8 +184,10 @@ int c2r_dispatch_dedup(const c2r_config* cfg, const int32_t* idx, const int32_t*
  * running under a host that forbids allocation on its hot path, or code in a latency-critical
  * section where cudaMalloc's device-wide synchronisation is not acceptable.
  *
- * Limit: ceil(N*K / 512) * E * 4 bytes must fit the array, i.e. about N*K <= 2.0 M slots at
- * E = 64; a larger batch is refused with C2R_ERR_STATIC_SCRATCH before anything is enqueued.
+ * Limit: ceil(N / b) * E * 4 bytes must fit the array, b = 512, 256, 160, 128, 96, 80, 64, 64 tokens
+ * for K = 1..8 (a block of the sort owns at most 512 slots), i.e. about N*K <= 2.0 M slots at
+ * E = 64 when K is a power of two; a larger batch is refused with C2R_ERR_STATIC_SCRATCH before
+ * anything is enqueued.
  * Cost: every GPU that loads the library carries the array (1 MiB) until the process exits.
  * Set-up: the first call on each device looks up the array's device address (with that device
  * current); make that first call outside any stream capture.
@@ -191,32 +210,42 @@ int c2r_pack_weights(const c2r_config* cfg, int n_experts, int I, const void* W1
 int c2r_unpack_weights(const c2r_config* cfg, int n_experts, int I, const void* W13p, void* W1,
                        void* W3, void* stream);
 
-/* Sec. 3.1 ("each token is fed to its selected experts"), expert = SwiGLU MLP without biases.
+/* Sec. 3.1: expert evaluation of the routed tokens; expert = SwiGLU MLP without biases.
  * For each expert e on rows [offsets[e], offsets[e]+counts[e]) of Xp:
- *   A = Xp W1_e^T, B = Xp W3_e^T, H = silu(A) * B, Yp = H W2_e^T.
+ *   A = Xp W1_e^T, B = Xp W3_e^T, H = s_r silu(A) * B, Yp = H W2_e^T,
+ * s_r the optional per-row scale (C2R_SCALE_*; row_scale [R] float, NULL with C2R_SCALE_NONE).  With the
+ * Eq. 1 weights as row scale, Yp already carries the weight of Sec. 3.1's weighted sum.
  * Xp [R,d] T; counts [n_experts], offsets [n_experts+1] int32 (device); W13p packed (above);
  * W2 [n_experts, d, I] T.  out: AB [R, 2I] T (what the backward pass needs from A and B, in the
- * packed column layout: the local derivatives dH/dA = B silu'(A) in the gate columns and
- * dH/dB = silu(A) in the up columns; AB == NULL skips it: forward only, e.g. inference),
- * H [R,I] T, Yp [R,d] float.
+ * packed column layout: the local derivatives B silu'(A) in the gate columns and silu(A) in the up
+ * columns, without the scale; AB == NULL skips it: forward only, e.g. inference),
+ * H [R,I] T (scale included), Yp [R,d] float.
  * R = rows of the buffers.  Padding rows of Xp must be zero.  n_experts = 1 with counts = {R},
  * offsets = {0,R} evaluates the dense shared expert.
  * bf16 runs on the tensor cores (tcgen05) when d % 16 == 0 and, for n_experts > 1, row_align is a
  * multiple of 128; other shapes and fp32 use a CUDA-core kernel.  status (one int32, may be NULL)
  * receives C2R_STATUS_WAIT_TIMEOUT if a bounded wait inside the kernel gave up (results invalid). */
 int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
-                           const int32_t* counts, const int32_t* offsets, const void* W13p,
-                           const void* W2, void* AB, void* H, void* Yp, int32_t* status, void* stream);
+                           const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
+                           const float* row_scale, int scale_kind, void* AB, void* H, void* Yp, int32_t* status,
+                           void* stream);
 
-/* Backward of the above:  dH = dYp W2; dA = dH * B * silu'(A); dB = dH * silu(A);
- * dXp = dA W1 + dB W3; dW2_e = dYp^T H; dW1_e = dA^T Xp; dW3_e = dB^T Xp.
- * dYp [R,d] T (padding rows zero); out: dAB [R,2I] T (packed columns), dXp [R,d] float,
- * dW13p [n_experts,2I,d] T (packed rows), dW2 [n_experts,d,I] T.  accumulate != 0 adds into the
- * weight gradients. */
+/* Backward of the above, given dYp = dLoss/dYp:  dH' = dYp W2 (the gradient w.r.t. the scaled H);
+ * dA = s_r dH' B silu'(A); dB = s_r dH' silu(A); dXp = dA W1 + dB W3; dW2_e = dYp^T H; dW1_e = dA^T Xp;
+ * dW3_e = dB^T Xp.  dYp [R,d] T (padding rows zero); AB, H as the forward call wrote them;
+ * out: dAB [R,2I] T (packed columns), dXp [R,d] float, dW13p [n_experts,2I,d] T (packed rows),
+ * dW2 [n_experts,d,I] T.  accumulate != 0 adds into the weight gradients.
+ * qpart (optional) [c2r_swiglu_qparts(...)][R] float: partial sums whose total over the first index is
+ * q_r = <dH'_r, H_r> = s_r dLoss/ds_r, the gradient w.r.t. the row's scale times the scale (added up in index
+ * order by c2r_route_bwd_scaled); rows outside every expert's segment are not written. */
 int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
-                           const int32_t* counts, const int32_t* offsets, const void* W13p,
-                           const void* W2, const void* AB, const void* H, const void* dYp, void* dAB,
-                           void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status, void* stream);
+                           const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
+                           const void* AB, const void* H, const void* dYp, const float* row_scale, int scale_kind,
+                           void* dAB, void* dXp, void* dW13p, void* dW2, float* qpart, int accumulate,
+                           int32_t* status, void* stream);
+
+/* First dimension of qpart for this shape (host function; -1 on a bad argument). */
+int c2r_swiglu_qparts(const c2r_config* cfg, int n_experts, int I, int64_t R);
 
 /* The two calls above with the dispatch folded into the GEMMs (an addition of this library: the gather-fused
  * form of the dispatch): wherever they read row r of Xp, the kernels read row slot_of_row[r] / K of X
@@ -226,17 +255,18 @@ int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t 
  * X [N,d] T; slot_of_row [R] int32 as c2r_permute wrote it. */
 int c2r_grouped_swiglu_fwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
                                   const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
-                                  const void* W13p, const void* W2, void* AB, void* H, void* Yp, int32_t* status,
-                                  void* stream);
+                                  const void* W13p, const void* W2, const float* row_scale, int scale_kind, void* AB,
+                                  void* H, void* Yp, int32_t* status, void* stream);
 int c2r_grouped_swiglu_bwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
                                   const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
                                   const void* W13p, const void* W2, const void* AB, const void* H, const void* dYp,
-                                  void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status,
-                                  void* stream);
+                                  const float* row_scale, int scale_kind, void* dAB, void* dXp, void* dW13p, void* dW2,
+                                  float* qpart, int accumulate, int32_t* status, void* stream);
 
 /* Sec. 3.1 (weighted sum of the selected experts' outputs):
  * Y[t,:] = sum_k w[t,k] * Yp[row_of_slot[t*K+k],:]  (k ascending, fp32)
  *          + sigmoid(z[t]) * Ys[t,:] when Ys != NULL (gated shared expert).
+ * w == NULL / z == NULL: that factor is 1 (the expert call already applied it as its row scale).
  * Yp [R,d] float; Ys [N,d] float; out: Y [N,d] T. */
 int c2r_combine(const c2r_config* cfg, const void* Yp, const float* w, const int32_t* row_of_slot,
                 const void* Ys, const float* z, void* Y, void* stream);
@@ -253,15 +283,25 @@ int c2r_combine_bwd(const c2r_config* cfg, const void* dY, const void* Yp, const
  * all other entries of dL are zero. */
 int c2r_route_bwd(const c2r_config* cfg, const float* w, const float* dw, float* dl, void* stream);
 
+/* c2r_route_bwd for experts that applied the weights themselves (C2R_SCALE_ROW / C2R_SCALE_SIGMOID): from the
+ * partial row dots the backward expert call left, q[t,k] = sum_j qpart[j, row_of_slot[t*K+k]] = w dLoss/dw,
+ *   dl[t,k] = q[t,k] - w[t,k] sum_j q[t,j]      (identical to the formula above, without dividing by w);
+ *   dw[t,k] = q[t,k] / w[t,k] (optional output, 0 where w is 0);
+ *   dz[t]   = (sum_j qspart[j,t]) (1 - sigmoid(z[t]))   (shared expert; optional).
+ * qpart [nq, c2r_permuted_rows] float; qspart [nqs, N] float. */
+int c2r_route_bwd_scaled(const c2r_config* cfg, const float* w, const int32_t* row_of_slot, const float* qpart, int nq,
+                         const float* z, const float* qspart, int nqs, float* dw, float* dl, float* dz, void* stream);
+
 /* Gate weight gradients: dWg[e,:] = sum_t dL[t,e] X[t,:], evaluated over expert e's rows of Xp
  * (dl addressed through slot_of_row); dwsg[:] = sum_t dz[t] X[t,:].
- * out: dWg [E,d] float; dwsg [d] float (iff dz != NULL).  ws: C2R_WS_GATE_BWD bytes.
+ * out: dWg [E,d] float; dwsg [d] float (iff dz != NULL); accumulate != 0 adds into both.
+ * ws: C2R_WS_GATE_BWD bytes.
  * bf16 with X and ws given: evaluated as one tensor-core GEMM dL^T X over a dense [N,64] bf16 copy of the
  * gradient w.r.t. the logits (dl and dz rounded to bf16, fp32 accumulation, token splits added in a fixed
  * order); otherwise a row-serial fp32 kernel over Xp. */
 int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
                  const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
-                 float* dWg, float* dwsg, void* ws, size_t ws_bytes, void* stream);
+                 float* dWg, float* dwsg, int accumulate, void* ws, size_t ws_bytes, void* stream);
 
 /* Gradient w.r.t. the hidden states (transpose of the dispatch, done as an atomic-free gather-sum):
  * dX[t,:] = sum_k dXp[row_of_slot[t*K+k],:]  + dXs[t,:]                (shared expert, optional)
@@ -305,13 +345,14 @@ typedef struct c2r_layer_buffers {
   int32_t* offsets;     /* [E+1] */
   int32_t* row_of_slot; /* [N*K] */
   int32_t* slot_of_row; /* [R] */
+  float* w_row;         /* [R]: w of the slot that owns each permuted row */
   void* Xp;             /* [R,d] */
   void* AB;             /* [R,2I]; NULL (with ABs) when no backward pass follows */
-  void* H;              /* [R,I] */
-  void* Yp;             /* [R,d] float */
+  void* H;              /* [R,I], Eq. 1 weight of the row included */
+  void* Yp;             /* [R,d] float, weight included */
   void* ABs;            /* [N,2I_s] */
-  void* Hs;             /* [N,I_s] */
-  void* Ys;             /* [N,d] float */
+  void* Hs;             /* [N,I_s], gate sigmoid(z) included */
+  void* Ys;             /* [N,d] float, gate included */
   int32_t* s_counts;    /* [1]  = {N}   (device) */
   int32_t* s_offsets;   /* [2]  = {0,N} (device) */
   void* Y;              /* [N,d] T: layer output */
@@ -319,13 +360,12 @@ typedef struct c2r_layer_buffers {
   int32_t* status;      /* one int32 */
   /* backward */
   const void* dY; /* [N,d] T */
-  void* dYp;      /* [R,d] */
+  void* dYp;      /* [R,d]: dY of the row's token */
   void* dAB;      /* [R,2I] */
   void* dXp;      /* [R,d] float */
-  void* dYs;      /* [N,d] */
   void* dABs;     /* [N,2I_s] */
   void* dXs;      /* [N,d] float */
-  float* dw;      /* [N,K] */
+  float* dw;      /* [N,K], may be NULL (informational: the backward pass itself needs only dl) */
   float* dl;      /* [N,K] */
   float* dz;      /* [N] */
   void* dW13p;    /* [E,2I,d] T */
@@ -339,17 +379,27 @@ typedef struct c2r_layer_buffers {
   int32_t* C;          /* [E,E] */
   int32_t* I_T;        /* [E,T] */
   uint64_t* mask_next; /* [E]: sets for the next step */
+  /* optional second stream for the shared expert, which depends on nothing the routing chain produces: a
+   * cudaStream_t and two cudaEvent_t (created with cudaEventDisableTiming) owned by the caller.  All three
+   * non-NULL: the shared expert's GEMMs are enqueued on stream2 between a fork from and a join into the
+   * drivers' stream, so they overlap gate -> route -> dispatch and fill the tails of the routed GEMMs. */
+  void* stream2;
+  void* ev_fork;
+  void* ev_join;
   /* scratch */
   void* ws;        /* C2R_WS_LAYER bytes */
   size_t ws_bytes;
 } c2r_layer_buffers;
 
-/* Forward of the whole layer on one stream, no host synchronisation:
+/* Forward of the whole layer, no host synchronisation:
  * gate -> route (C2R or Top-K) -> permute -> grouped SwiGLU (+ shared expert) -> combine
- * (-> dispatch volume when part != NULL). */
+ * (-> dispatch volume when part != NULL).  The Eq. 1 weights and the shared expert's gate are applied
+ * inside the expert calls (row scale), so the combine is a plain sum. */
 int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, void* stream);
 
-/* Backward of c2r_layer_fwd (routing decision frozen) using the state it left in `b`. */
+/* Backward of c2r_layer_fwd (routing decision frozen) using the state it left in `b`.
+ * accumulate != 0 adds into every parameter gradient (dW13p, dW2, dWs13p, dWs2, dWg, dwsg); dX is always
+ * overwritten. */
 int c2r_layer_bwd(const c2r_config* cfg, const c2r_layer_buffers* b, int accumulate, void* stream);
 
 /* Forward, backward, then Eq. 2 and Eq. 4 on this step's routing: C is overwritten from idx and

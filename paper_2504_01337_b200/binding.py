@@ -39,11 +39,11 @@ class Config(C.Structure):
 
 _LAYER_FIELDS = [
     "X", "Wg", "wsg", "W13p", "W2", "Ws13p", "Ws2", "mask", "expert_rank", "part",
-    "L", "z", "idx", "w", "counts", "offsets", "row_of_slot", "slot_of_row", "Xp", "AB", "H", "Yp",
+    "L", "z", "idx", "w", "counts", "offsets", "row_of_slot", "slot_of_row", "w_row", "Xp", "AB", "H", "Yp",
     "ABs", "Hs", "Ys", "s_counts", "s_offsets", "Y", "volume", "status",
-    "dY", "dYp", "dAB", "dXp", "dYs", "dABs", "dXs", "dw", "dl", "dz",
+    "dY", "dYp", "dAB", "dXp", "dABs", "dXs", "dw", "dl", "dz",
     "dW13p", "dW2", "dWs13p", "dWs2", "dWg", "dwsg", "dX",
-    "C", "I_T", "mask_next", "ws",
+    "C", "I_T", "mask_next", "stream2", "ev_fork", "ev_join", "ws",
 ]
 
 
@@ -57,7 +57,8 @@ EXPORTS = [
     "c2r_unpack_weights", "c2r_grouped_swiglu_fwd", "c2r_grouped_swiglu_bwd", "c2r_combine", "c2r_combine_bwd",
     "c2r_route_bwd", "c2r_gate_bwd", "c2r_unpermute_grad", "c2r_dispatch_volume", "c2r_layer_fwd",
     "c2r_layer_bwd", "c2r_train_step", "c2r_permute_static", "c2r_dispatch_dedup",
-    "c2r_grouped_swiglu_fwd_gather", "c2r_grouped_swiglu_bwd_gather",
+    "c2r_grouped_swiglu_fwd_gather", "c2r_grouped_swiglu_bwd_gather", "c2r_permute_rows", "c2r_swiglu_qparts",
+    "c2r_route_bwd_scaled",
 ]
 
 _P = C.c_void_p
@@ -70,24 +71,27 @@ lib.c2r_last_cuda_error.restype = C.c_int
 lib.c2r_launch_count.restype = C.c_uint64
 _SIGS = {
     "c2r_gate_logits": [_CFG] + [_P] * 6,
-    "c2r_route": [_CFG] + [_P] * 7,
+    "c2r_route": [_CFG] + [_P] * 8,
     "c2r_collab_count": [_CFG, _P, C.c_int64, _P, C.c_int, _P],
     "c2r_collab_sets": [_CFG] + [_P] * 4,
     "c2r_collab_degree": [_CFG] + [_P] * 4,
     "c2r_place_experts": [_CFG, _P, C.c_int, _P, _P],
-    "c2r_permute": [_CFG] + [_P] * 10 + [C.c_size_t, _P],
+    "c2r_permute": [_CFG] + [_P] * 12 + [C.c_size_t, C.c_int, _P],
+    "c2r_permute_rows": [_CFG] + [_P] * 6,
+    "c2r_swiglu_qparts": [_CFG, C.c_int, C.c_int, C.c_int64],
+    "c2r_route_bwd_scaled": [_CFG, _P, _P, _P, C.c_int, _P, _P, C.c_int, _P, _P, _P, _P],
     "c2r_permute_static": [_CFG] + [_P] * 10,
     "c2r_dispatch_dedup": [_CFG] + [_P] * 16 + [C.c_size_t, _P],
     "c2r_pack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
     "c2r_unpack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
-    "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 10,
-    "c2r_grouped_swiglu_bwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 12 + [C.c_int, _P, _P],
-    "c2r_grouped_swiglu_fwd_gather": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 11,
-    "c2r_grouped_swiglu_bwd_gather": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 13 + [C.c_int, _P, _P],
+    "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 6 + [C.c_int] + [_P] * 5,
+    "c2r_grouped_swiglu_bwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 9 + [C.c_int] + [_P] * 5 + [C.c_int, _P, _P],
+    "c2r_grouped_swiglu_fwd_gather": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 7 + [C.c_int] + [_P] * 5,
+    "c2r_grouped_swiglu_bwd_gather": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 10 + [C.c_int] + [_P] * 5 + [C.c_int, _P, _P],
     "c2r_combine": [_CFG] + [_P] * 7,
     "c2r_combine_bwd": [_CFG] + [_P] * 12,
     "c2r_route_bwd": [_CFG] + [_P] * 4,
-    "c2r_gate_bwd": [_CFG] + [_P] * 10 + [C.c_size_t, _P],
+    "c2r_gate_bwd": [_CFG] + [_P] * 9 + [C.c_int, _P, C.c_size_t, _P],
     "c2r_unpermute_grad": [_CFG] + [_P] * 9 + [C.c_int, _P],
     "c2r_dispatch_volume": [_CFG] + [_P] * 6,
     "c2r_layer_fwd": [_CFG, C.POINTER(LayerBuffers), _P],
@@ -100,6 +104,7 @@ for _name, _sig in _SIGS.items():
 
 
 FLAG_GATHER_FUSED = 1
+SCALE_NONE, SCALE_ROW, SCALE_SIGMOID = 0, 1, 2
 
 
 def make_config(N, d, E, I, K, T=0, P=1, I_s=0, dtype=BF16, row_align=1, renorm=1, flags=0) -> Config:
@@ -149,8 +154,9 @@ def gate_logits(cfg, X, Wg, wsg, L, z):
     _call("c2r_gate_logits", C.byref(cfg), _ptr(X), _ptr(Wg), _ptr(wsg), _ptr(L), _ptr(z), _stream())
 
 
-def route(cfg, L, mask, idx, w, p=None, status=None):
-    _call("c2r_route", C.byref(cfg), _ptr(L), _ptr(mask), _ptr(idx), _ptr(w), _ptr(p), _ptr(status), _stream())
+def route(cfg, L, mask, idx, w, p=None, status=None, permute_ws=None):
+    _call("c2r_route", C.byref(cfg), _ptr(L), _ptr(mask), _ptr(idx), _ptr(w), _ptr(p), _ptr(status), _ptr(permute_ws),
+          _stream())
 
 
 def collab_count(cfg, idx, n_tokens, Cmat, accumulate=False):
@@ -169,10 +175,27 @@ def place_experts(cfg, C_host, mode, part_host, rank_host):
     _call("c2r_place_experts", C.byref(cfg), _host_ptr(C_host), int(mode), _host_ptr(part_host), _host_ptr(rank_host))
 
 
-def permute(cfg, idx, expert_rank, X, counts, offsets, row_of_slot, slot_of_row, Xp, status, ws):
-    _call("c2r_permute", C.byref(cfg), _ptr(idx), _ptr(expert_rank), _ptr(X), _ptr(counts), _ptr(offsets),
-          _ptr(row_of_slot), _ptr(slot_of_row), _ptr(Xp), _ptr(status), _ptr(ws),
-          0 if ws is None else ws.numel() * ws.element_size(), _stream())
+def permute(cfg, idx, expert_rank, X, counts, offsets, row_of_slot, slot_of_row, Xp, status, ws, w=None, w_row=None,
+            ws_has_histogram=False):
+    _call("c2r_permute", C.byref(cfg), _ptr(idx), _ptr(expert_rank), _ptr(X), _ptr(w), _ptr(counts), _ptr(offsets),
+          _ptr(row_of_slot), _ptr(slot_of_row), _ptr(Xp), _ptr(w_row), _ptr(status), _ptr(ws),
+          0 if ws is None else ws.numel() * ws.element_size(), int(ws_has_histogram), _stream())
+
+
+def permute_rows(cfg, X, row_of_slot, counts, offsets, Xp):
+    _call("c2r_permute_rows", C.byref(cfg), _ptr(X), _ptr(row_of_slot), _ptr(counts), _ptr(offsets), _ptr(Xp), _stream())
+
+
+def swiglu_qparts(cfg, n_experts, I, R):
+    n = int(lib.c2r_swiglu_qparts(C.byref(cfg), n_experts, I, int(R)))
+    if n < 0:
+        raise C2RError("c2r_swiglu_qparts", -1)
+    return n
+
+
+def route_bwd_scaled(cfg, w, row_of_slot, qpart, nq, z, qspart, nqs, dw, dl, dz):
+    _call("c2r_route_bwd_scaled", C.byref(cfg), _ptr(w), _ptr(row_of_slot), _ptr(qpart), int(nq), _ptr(z), _ptr(qspart),
+          int(nqs), _ptr(dw), _ptr(dl), _ptr(dz), _stream())
 
 
 def permute_static(cfg, idx, expert_rank, X, counts, offsets, row_of_slot, slot_of_row, Xp, status):
@@ -197,28 +220,37 @@ def unpack_weights(cfg, n_experts, I, W13p, W1, W3):
     _call("c2r_unpack_weights", C.byref(cfg), n_experts, I, _ptr(W13p), _ptr(W1), _ptr(W3), _stream())
 
 
-def grouped_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, status=None):
+def _scale_kind(row_scale, scale_kind):
+    return SCALE_NONE if row_scale is None else int(scale_kind)
+
+
+def grouped_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, status=None, row_scale=None,
+                       scale_kind=SCALE_ROW):
     _call("c2r_grouped_swiglu_fwd", C.byref(cfg), n_experts, I, int(R), _ptr(Xp), _ptr(counts), _ptr(offsets),
-          _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(Yp), _ptr(status), _stream())
+          _ptr(W13p), _ptr(W2), _ptr(row_scale), _scale_kind(row_scale, scale_kind), _ptr(AB), _ptr(H), _ptr(Yp),
+          _ptr(status), _stream())
 
 
 def grouped_swiglu_bwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p, dW2,
-                       accumulate=False, status=None):
+                       accumulate=False, status=None, row_scale=None, scale_kind=SCALE_ROW, qpart=None):
     _call("c2r_grouped_swiglu_bwd", C.byref(cfg), n_experts, I, int(R), _ptr(Xp), _ptr(counts), _ptr(offsets),
-          _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2),
-          int(accumulate), _ptr(status), _stream())
+          _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(row_scale), _scale_kind(row_scale, scale_kind),
+          _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2), _ptr(qpart), int(accumulate), _ptr(status), _stream())
 
 
-def grouped_swiglu_fwd_gather(cfg, n_experts, I, R, X, slot_of_row, counts, offsets, W13p, W2, AB, H, Yp, status=None):
+def grouped_swiglu_fwd_gather(cfg, n_experts, I, R, X, slot_of_row, counts, offsets, W13p, W2, AB, H, Yp, status=None,
+                              row_scale=None, scale_kind=SCALE_ROW):
     _call("c2r_grouped_swiglu_fwd_gather", C.byref(cfg), n_experts, I, int(R), _ptr(X), _ptr(slot_of_row), _ptr(counts),
-          _ptr(offsets), _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(Yp), _ptr(status), _stream())
+          _ptr(offsets), _ptr(W13p), _ptr(W2), _ptr(row_scale), _scale_kind(row_scale, scale_kind), _ptr(AB), _ptr(H),
+          _ptr(Yp), _ptr(status), _stream())
 
 
 def grouped_swiglu_bwd_gather(cfg, n_experts, I, R, X, slot_of_row, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p,
-                              dW2, accumulate=False, status=None):
+                              dW2, accumulate=False, status=None, row_scale=None, scale_kind=SCALE_ROW, qpart=None):
     _call("c2r_grouped_swiglu_bwd_gather", C.byref(cfg), n_experts, I, int(R), _ptr(X), _ptr(slot_of_row), _ptr(counts),
-          _ptr(offsets), _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2),
-          int(accumulate), _ptr(status), _stream())
+          _ptr(offsets), _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(row_scale),
+          _scale_kind(row_scale, scale_kind), _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2), _ptr(qpart), int(accumulate),
+          _ptr(status), _stream())
 
 
 def combine(cfg, Yp, w, row_of_slot, Ys, z, Y):
@@ -234,9 +266,10 @@ def route_bwd(cfg, w, dw, dl):
     _call("c2r_route_bwd", C.byref(cfg), _ptr(w), _ptr(dw), _ptr(dl), _stream())
 
 
-def gate_bwd(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws):
+def gate_bwd(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws, accumulate=False):
     _call("c2r_gate_bwd", C.byref(cfg), _ptr(X), _ptr(Xp), _ptr(counts), _ptr(offsets), _ptr(slot_of_row), _ptr(dl),
-          _ptr(dz), _ptr(dWg), _ptr(dwsg), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(), _stream())
+          _ptr(dz), _ptr(dWg), _ptr(dwsg), int(accumulate), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+          _stream())
 
 
 def unpermute_grad(cfg, dXp, row_of_slot, dXs, idx, dl, Wg, dz, wsg, dX, accumulate=False):
@@ -254,6 +287,10 @@ def make_layer_buffers(tensors: dict) -> LayerBuffers:
     b = LayerBuffers()
     for name in _LAYER_FIELDS:
         t = tensors.get(name)
+        if name == "stream2":
+            t = None if t is None else t.cuda_stream
+        elif name in ("ev_fork", "ev_join"):
+            t = None if t is None else t.cuda_event
         setattr(b, name, _ptr(t))
     ws = tensors.get("ws")
     b.ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()

@@ -19,7 +19,7 @@ extern "C" size_t c2r_workspace_bytes(const c2r_config* cfg, int which) {
   switch (which) {
     case C2R_WS_PERMUTE: return align256(permute_ws_bytes(cfg));
     case C2R_WS_GATE_BWD: return align256(gate_bwd_ws_bytes(cfg));
-    case C2R_WS_LAYER: return align256(permute_ws_bytes(cfg)) + align256(gate_bwd_ws_bytes(cfg));
+    case C2R_WS_LAYER: return layer_ws_bytes(cfg);
     case C2R_WS_DISPATCH_DEDUP: return align256(dispatch_dedup_ws_bytes(cfg));
     default: return 0;
   }
@@ -71,66 +71,100 @@ static int check_gemm_args(const c2r_config* cfg, int nE, int I, int64_t R) {
   return C2R_OK;
 }
 
+static int check_scale(const float* row_scale, int scale_kind) {
+  C2R_REQUIRE(scale_kind == C2R_SCALE_NONE || scale_kind == C2R_SCALE_ROW || scale_kind == C2R_SCALE_SIGMOID,
+              C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(scale_kind == C2R_SCALE_NONE || row_scale != nullptr, C2R_ERR_INVALID_ARG);
+  return C2R_OK;
+}
+
+static int swiglu_fwd_dispatch(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
+  if (a.R == 0) return C2R_OK;
+  if (cfg->dtype == C2R_F32) return simt_swiglu_fwd<float>(cfg, a, s);
+  if (tc_supported(cfg, a.nE, a.I, a.R)) return tc_swiglu_fwd(cfg, a, s);
+  return simt_swiglu_fwd<__nv_bfloat16>(cfg, a, s);
+}
+
+static int swiglu_bwd_dispatch(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
+  if (a.R == 0) return C2R_OK;
+  if (cfg->dtype == C2R_F32) return simt_swiglu_bwd<float>(cfg, a, s);
+  if (tc_supported(cfg, a.nE, a.I, a.R)) return tc_swiglu_bwd(cfg, a, s);
+  return simt_swiglu_bwd<__nv_bfloat16>(cfg, a, s);
+}
+
+extern "C" int c2r_swiglu_qparts(const c2r_config* cfg, int n_experts, int I, int64_t R) {
+  if (check_gemm_args(cfg, n_experts, I, R) != C2R_OK) return -1;
+  return swiglu_qparts(cfg, n_experts, I, R);
+}
+
 extern "C" int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                                       const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
-                                      void* AB, void* H, void* Yp, int32_t* status, void* stream) {
+                                      const float* row_scale, int scale_kind, void* AB, void* H, void* Yp,
+                                      int32_t* status, void* stream) {
   int rc = check_gemm_args(cfg, n_experts, I, R);
   if (rc) return rc;
   C2R_REQUIRE(Xp && counts && offsets && W13p && W2 && H && Yp, C2R_ERR_INVALID_ARG);
-  if (R == 0) return C2R_OK;
-  cudaStream_t s = as_stream(stream);
-  if (cfg->dtype == C2R_F32) {
-    return simt_swiglu_fwd<float>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, s);
-  }
-  if (tc_supported(cfg, n_experts, I, R))
-    return tc_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, status, s);
-  return simt_swiglu_fwd<__nv_bfloat16>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, s);
+  if ((rc = check_scale(row_scale, scale_kind))) return rc;
+  SwigluCall a{};
+  a.nE = n_experts; a.I = I; a.R = R; a.Xp = Xp; a.counts = counts; a.offsets = offsets; a.W13p = W13p; a.W2 = W2;
+  a.row_scale = row_scale; a.scale_kind = scale_kind; a.AB = AB; a.H = H; a.Yp = Yp; a.status = status;
+  return swiglu_fwd_dispatch(cfg, a, as_stream(stream));
 }
 
 extern "C" int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                                       const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
-                                      const void* AB, const void* H, const void* dYp, void* dAB, void* dXp,
-                                      void* dW13p, void* dW2, int accumulate, int32_t* status, void* stream) {
+                                      const void* AB, const void* H, const void* dYp, const float* row_scale,
+                                      int scale_kind, void* dAB, void* dXp, void* dW13p, void* dW2, float* qpart,
+                                      int accumulate, int32_t* status, void* stream) {
   int rc = check_gemm_args(cfg, n_experts, I, R);
   if (rc) return rc;
   C2R_REQUIRE(Xp && counts && offsets && W13p && W2 && AB && H && dYp && dAB && dXp && dW13p && dW2,
               C2R_ERR_INVALID_ARG);
-  cudaStream_t s = as_stream(stream);
-  if (cfg->dtype == C2R_F32)
-    return simt_swiglu_bwd<float>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p,
-                                  dW2, accumulate, s);
-  if (tc_supported(cfg, n_experts, I, R))
-    return tc_swiglu_bwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p, dW2,
-                         accumulate, status, s);
-  return simt_swiglu_bwd<__nv_bfloat16>(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp,
-                                        dW13p, dW2, accumulate, s);
+  if ((rc = check_scale(row_scale, scale_kind))) return rc;
+  SwigluCall a{};
+  a.nE = n_experts; a.I = I; a.R = R; a.Xp = Xp; a.counts = counts; a.offsets = offsets; a.W13p = W13p; a.W2 = W2;
+  a.row_scale = row_scale; a.scale_kind = scale_kind; a.AB = const_cast<void*>(AB); a.H = const_cast<void*>(H);
+  a.dYp = dYp; a.dAB = dAB; a.dXp = dXp; a.dW13p = dW13p; a.dW2 = dW2; a.qpart = qpart; a.accumulate = accumulate;
+  a.status = status;
+  return swiglu_bwd_dispatch(cfg, a, as_stream(stream));
 }
 
 extern "C" int c2r_grouped_swiglu_fwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
                                              const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
-                                             const void* W13p, const void* W2, void* AB, void* H, void* Yp,
-                                             int32_t* status, void* stream) {
+                                             const void* W13p, const void* W2, const float* row_scale, int scale_kind,
+                                             void* AB, void* H, void* Yp, int32_t* status, void* stream) {
   int rc = check_gemm_args(cfg, n_experts, I, R);
   if (rc) return rc;
   C2R_REQUIRE(X && slot_of_row && counts && offsets && W13p && W2 && H && Yp, C2R_ERR_INVALID_ARG);
+  if ((rc = check_scale(row_scale, scale_kind))) return rc;
   C2R_REQUIRE(tc_supported(cfg, n_experts, I, R) && (((uintptr_t)X) & 15u) == 0, C2R_ERR_UNSUPPORTED_SHAPE);
   if (R == 0) return C2R_OK;
-  return tc_swiglu_fwd(cfg, n_experts, I, R, nullptr, counts, offsets, W13p, W2, AB, H, Yp, status, as_stream(stream), X,
-                       slot_of_row);
+  SwigluCall a{};
+  a.nE = n_experts; a.I = I; a.R = R; a.counts = counts; a.offsets = offsets; a.W13p = W13p; a.W2 = W2;
+  a.row_scale = row_scale; a.scale_kind = scale_kind; a.AB = AB; a.H = H; a.Yp = Yp; a.status = status;
+  a.X = X; a.slot_of_row = slot_of_row;
+  return tc_swiglu_fwd(cfg, a, as_stream(stream));
 }
 
 extern "C" int c2r_grouped_swiglu_bwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
                                              const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
                                              const void* W13p, const void* W2, const void* AB, const void* H,
-                                             const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2,
-                                             int accumulate, int32_t* status, void* stream) {
+                                             const void* dYp, const float* row_scale, int scale_kind, void* dAB,
+                                             void* dXp, void* dW13p, void* dW2, float* qpart, int accumulate,
+                                             int32_t* status, void* stream) {
   int rc = check_gemm_args(cfg, n_experts, I, R);
   if (rc) return rc;
   C2R_REQUIRE(X && slot_of_row && counts && offsets && W13p && W2 && AB && H && dYp && dAB && dXp && dW13p && dW2,
               C2R_ERR_INVALID_ARG);
+  if ((rc = check_scale(row_scale, scale_kind))) return rc;
   C2R_REQUIRE(tc_supported(cfg, n_experts, I, R) && (((uintptr_t)X) & 15u) == 0, C2R_ERR_UNSUPPORTED_SHAPE);
-  return tc_swiglu_bwd(cfg, n_experts, I, R, nullptr, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p, dW2, accumulate,
-                       status, as_stream(stream), X, slot_of_row);
+  if (R == 0) return C2R_OK;
+  SwigluCall a{};
+  a.nE = n_experts; a.I = I; a.R = R; a.counts = counts; a.offsets = offsets; a.W13p = W13p; a.W2 = W2;
+  a.row_scale = row_scale; a.scale_kind = scale_kind; a.AB = const_cast<void*>(AB); a.H = const_cast<void*>(H);
+  a.dYp = dYp; a.dAB = dAB; a.dXp = dXp; a.dW13p = dW13p; a.dW2 = dW2; a.qpart = qpart; a.accumulate = accumulate;
+  a.status = status; a.X = X; a.slot_of_row = slot_of_row;
+  return tc_swiglu_bwd(cfg, a, as_stream(stream));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -148,32 +182,90 @@ static bool gather_fused(const c2r_config* cfg, const void* X) {
          cfg->E < 64 && tc_supported(cfg, cfg->E, cfg->I, permuted_rows(cfg));
 }
 
+// Layout of the C2R_WS_LAYER workspace.
+struct LayerWs {
+  char* permute;    // per-block expert counts of the dispatch
+  char* gate_bwd;   // scratch of c2r_gate_bwd
+  float* qpart;     // [nq][R] partial row dots of the routed experts' backward
+  float* qspart;    // [nqs][N] the same for the shared expert
+  int nq, nqs;
+  size_t bytes;
+};
+static LayerWs layer_ws(const c2r_config* cfg, void* base) {
+  LayerWs w;
+  const int64_t R = permuted_rows(cfg);
+  w.nq = swiglu_qparts(cfg, cfg->E, cfg->I > 0 ? cfg->I : 16, R);
+  w.nqs = cfg->I_s > 0 ? swiglu_qparts(cfg, 1, cfg->I_s, cfg->N) : 0;
+  size_t o = 0;
+  w.permute = (char*)base + o; o += align256(permute_ws_bytes(cfg));
+  w.gate_bwd = (char*)base + o; o += align256(gate_bwd_ws_bytes(cfg));
+  w.qpart = (float*)((char*)base + o); o += align256(sizeof(float) * (size_t)w.nq * (size_t)R);
+  w.qspart = (float*)((char*)base + o); o += align256(sizeof(float) * (size_t)w.nqs * (size_t)cfg->N);
+  w.bytes = o;
+  return w;
+}
+size_t c2r::layer_ws_bytes(const c2r_config* cfg) { return layer_ws(cfg, nullptr).bytes; }
+
+// The shared expert depends on nothing the routing chain produces.  With a second stream (and two events) in the
+// buffers its GEMMs are enqueued there, between fork() and join(); without, everything stays on the one stream.
+struct SideStream {
+  cudaStream_t main, side;
+  cudaEvent_t fork_ev, join_ev;
+  bool on;
+  SideStream(const c2r_layer_buffers* b, void* stream, bool wanted)
+      : main(as_stream(stream)), side((cudaStream_t)b->stream2), fork_ev((cudaEvent_t)b->ev_fork),
+        join_ev((cudaEvent_t)b->ev_join), on(wanted && b->stream2 && b->ev_fork && b->ev_join) {}
+  void* work() const { return on ? (void*)side : (void*)main; }
+  int fork() const {
+    if (!on) return C2R_OK;
+    C2R_CUDA(cudaEventRecord(fork_ev, main));
+    C2R_CUDA(cudaStreamWaitEvent(side, fork_ev, 0));
+    return C2R_OK;
+  }
+  int join() const {
+    if (!on) return C2R_OK;
+    C2R_CUDA(cudaEventRecord(join_ev, side));
+    C2R_CUDA(cudaStreamWaitEvent(main, join_ev, 0));
+    return C2R_OK;
+  }
+};
+
 extern "C" int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   C2R_REQUIRE(b, C2R_ERR_INVALID_ARG);
   const bool shared = cfg->I_s > 0;
   C2R_REQUIRE(b->ws && b->ws_bytes >= c2r_workspace_bytes(cfg, C2R_WS_LAYER), C2R_ERR_WORKSPACE);
+  C2R_REQUIRE(b->w_row, C2R_ERR_INVALID_ARG);
   if (shared)
     C2R_REQUIRE(b->wsg && b->z && b->Ws13p && b->Ws2 && b->Hs && b->Ys && b->s_counts && b->s_offsets,
                 C2R_ERR_INVALID_ARG);
   const int64_t R = permuted_rows(cfg);
+  const LayerWs ws = layer_ws(cfg, b->ws);
+  const SideStream ss(b, stream, shared);
   C2R_TRY(gate_logits_impl(cfg, b->X, b->Wg, shared ? b->wsg : nullptr, b->L, b->z, b->status, stream));
-  C2R_TRY(c2r_route(cfg, b->L, b->mask, b->idx, b->w, nullptr, b->status, stream));
+  if (shared) {
+    // shared expert, its sigmoid gate applied to H inside the GEMM: Ys = sigmoid(z) * Shared(x)
+    C2R_TRY(ss.fork());
+    C2R_TRY(c2r_grouped_swiglu_fwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->z,
+                                   C2R_SCALE_SIGMOID, b->ABs, b->Hs, b->Ys, b->status, ss.work()));
+  }
+  // routing leaves the dispatch's per-block histogram in the workspace; the dispatch also spreads the weights
+  C2R_TRY(route_impl(cfg, b->L, b->mask, b->idx, b->w, nullptr, b->status, (int32_t*)ws.permute, stream));
   const bool fused = gather_fused(cfg, b->X);
-  C2R_TRY(c2r_permute(cfg, b->idx, b->expert_rank, fused ? nullptr : b->X, b->counts, b->offsets, b->row_of_slot,
-                      b->slot_of_row, b->Xp, b->status, b->ws, b->ws_bytes, stream));
+  C2R_TRY(permute_call(cfg, b->idx, b->expert_rank, fused ? nullptr : b->X, b->counts, b->offsets, b->row_of_slot,
+                       b->slot_of_row, b->Xp, b->status, ws.permute, align256(permute_ws_bytes(cfg)), stream, cfg->N > 0,
+                       b->w, b->w_row));
+  // routed experts with the Eq. 1 weight of each row applied to H: Yp = w * Expert(x)
   if (fused)
     C2R_TRY(c2r_grouped_swiglu_fwd_gather(cfg, cfg->E, cfg->I, R, b->X, b->slot_of_row, b->counts, b->offsets, b->W13p,
-                                          b->W2, b->AB, b->H, b->Yp, b->status, stream));
+                                          b->W2, b->w_row, C2R_SCALE_ROW, b->AB, b->H, b->Yp, b->status, stream));
   else
-    C2R_TRY(c2r_grouped_swiglu_fwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
-                                   b->Yp, b->status, stream));
-  if (shared)
-    C2R_TRY(c2r_grouped_swiglu_fwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
-                                   b->Hs, b->Ys, b->status, stream));
-  C2R_TRY(c2r_combine(cfg, b->Yp, b->w, b->row_of_slot, shared ? b->Ys : nullptr, shared ? b->z : nullptr, b->Y,
-                      stream));
+    C2R_TRY(c2r_grouped_swiglu_fwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->w_row,
+                                   C2R_SCALE_ROW, b->AB, b->H, b->Yp, b->status, stream));
+  C2R_TRY(ss.join());
+  // the weights are already inside Yp and Ys: a plain sum over the token's K rows plus the shared term
+  C2R_TRY(c2r_combine(cfg, b->Yp, nullptr, b->row_of_slot, shared ? b->Ys : nullptr, nullptr, b->Y, stream));
   if (b->part && b->volume) {
     const int P = cfg->P;
     C2R_TRY(c2r_dispatch_volume(cfg, b->idx, b->part, b->volume, b->volume + 4, b->volume + 4 + P * P, stream));
@@ -187,28 +279,35 @@ extern "C" int c2r_layer_bwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
   C2R_REQUIRE(b, C2R_ERR_INVALID_ARG);
   const bool shared = cfg->I_s > 0;
   C2R_REQUIRE(b->ws && b->ws_bytes >= c2r_workspace_bytes(cfg, C2R_WS_LAYER), C2R_ERR_WORKSPACE);
-  C2R_REQUIRE(b->dY && b->dYp && b->dAB && b->dXp && b->dw && b->dl && b->dW13p && b->dW2 && b->dWg && b->dX,
+  C2R_REQUIRE(b->dY && b->dYp && b->dAB && b->dXp && b->dl && b->dW13p && b->dW2 && b->dWg && b->dX && b->w_row,
               C2R_ERR_INVALID_ARG);
-  if (shared)
-    C2R_REQUIRE(b->dYs && b->dABs && b->dXs && b->dz && b->dWs13p && b->dWs2 && b->dwsg, C2R_ERR_INVALID_ARG);
+  if (shared) C2R_REQUIRE(b->dABs && b->dXs && b->dz && b->dWs13p && b->dWs2 && b->dwsg, C2R_ERR_INVALID_ARG);
   const int64_t R = permuted_rows(cfg);
-  char* ws_gate = (char*)b->ws + align256(permute_ws_bytes(cfg));
-  C2R_TRY(c2r_combine_bwd(cfg, b->dY, b->Yp, b->w, b->row_of_slot, b->slot_of_row, shared ? b->Ys : nullptr,
-                          shared ? b->z : nullptr, b->dYp, b->dw, shared ? b->dYs : nullptr,
-                          shared ? b->dz : nullptr, stream));
+  const LayerWs ws = layer_ws(cfg, b->ws);
+  const SideStream ss(b, stream, shared);
+  if (shared) {
+    // the shared expert reads dY as it is; its gate enters through the row scale
+    C2R_TRY(ss.fork());
+    C2R_TRY(c2r_grouped_swiglu_bwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
+                                   b->Hs, b->dY, b->z, C2R_SCALE_SIGMOID, b->dABs, b->dXs, b->dWs13p, b->dWs2, ws.qspart,
+                                   accumulate, b->status, ss.work()));
+  }
+  // transpose of the combine's gather: every permuted row receives its token's dY unchanged
+  C2R_TRY(c2r_permute_rows(cfg, b->dY, b->row_of_slot, b->counts, b->offsets, b->dYp, stream));
   if (gather_fused(cfg, b->X))
     C2R_TRY(c2r_grouped_swiglu_bwd_gather(cfg, cfg->E, cfg->I, R, b->X, b->slot_of_row, b->counts, b->offsets, b->W13p,
-                                          b->W2, b->AB, b->H, b->dYp, b->dAB, b->dXp, b->dW13p, b->dW2, accumulate,
-                                          b->status, stream));
+                                          b->W2, b->AB, b->H, b->dYp, b->w_row, C2R_SCALE_ROW, b->dAB, b->dXp, b->dW13p,
+                                          b->dW2, ws.qpart, accumulate, b->status, stream));
   else
     C2R_TRY(c2r_grouped_swiglu_bwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
-                                   b->dYp, b->dAB, b->dXp, b->dW13p, b->dW2, accumulate, b->status, stream));
-  if (shared)
-    C2R_TRY(c2r_grouped_swiglu_bwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
-                                   b->Hs, b->dYs, b->dABs, b->dXs, b->dWs13p, b->dWs2, accumulate, b->status, stream));
-  C2R_TRY(c2r_route_bwd(cfg, b->w, b->dw, b->dl, stream));
+                                   b->dYp, b->w_row, C2R_SCALE_ROW, b->dAB, b->dXp, b->dW13p, b->dW2, ws.qpart, accumulate,
+                                   b->status, stream));
+  C2R_TRY(ss.join());
+  C2R_TRY(c2r_route_bwd_scaled(cfg, b->w, b->row_of_slot, ws.qpart, ws.nq, shared ? b->z : nullptr, ws.qspart, ws.nqs, b->dw,
+                               b->dl, shared ? b->dz : nullptr, stream));
   C2R_TRY(c2r_gate_bwd(cfg, b->X, b->Xp, b->counts, b->offsets, b->slot_of_row, b->dl, shared ? b->dz : nullptr,
-                       b->dWg, shared ? b->dwsg : nullptr, ws_gate, align256(gate_bwd_ws_bytes(cfg)), stream));
+                       b->dWg, shared ? b->dwsg : nullptr, accumulate, ws.gate_bwd, align256(gate_bwd_ws_bytes(cfg)),
+                       stream));
   C2R_TRY(c2r_unpermute_grad(cfg, b->dXp, b->row_of_slot, shared ? b->dXs : nullptr, b->idx, b->dl, b->Wg,
                              shared ? b->dz : nullptr, shared ? b->wsg : nullptr, b->dX, 0, stream));
   return C2R_OK;

@@ -52,6 +52,13 @@ inline int64_t permuted_rows(const c2r_config* c) {
   return round_up((int64_t)c->N * c->K + (int64_t)c->E * (c->row_align - 1), c->row_align);
 }
 
+// Tokens owned by one block of the dispatch's counting sort: the largest count that keeps a block at no
+// more than 512 slots and a whole number of 32-slot groups (K = 1, 2, 4, 8: exactly 512 slots).
+__host__ __device__ inline int perm_tokens_per_block(int K) {
+  const int m = 32 / (K & -K);  // tokens per whole number of 32-slot groups (K <= 8)
+  return (512 / K) / m * m;
+}
+
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
 // ---- device helpers -------------------------------------------------------------------------

@@ -22,34 +22,59 @@ struct SimtGemm {
   void* C;
   const void* aux;
   void* aux_out;
+  const void* aux2;        // SIMT_EPI_SWIGLU_BWD: the forward's H (for the row dots), or NULL
+  const float* row_scale;  // SwiGLU forms: per-row scale of H, see SwigluCall
+  int scale_kind;
+  float* qpart;            // SIMT_EPI_SWIGLU_BWD: [ceil(I / 64)][R] partial row dots, or NULL
+  long long R;
   const int32_t* counts;
   const int32_t* offsets;
   long long sam, sak, sbn, sbk, sB, sC, ldc;
   int mode, epi, Mdim, Ndim, Kdim, I, accumulate;
 };
 
+// One grouped SwiGLU evaluation (forward or backward); members a direction does not use stay NULL.
+// Per-row scale: H = s_r silu(A) B with s_r = 1 (kind C2R_SCALE_NONE), row_scale[r] (C2R_SCALE_ROW) or
+// sigmoid(row_scale[r]) (C2R_SCALE_SIGMOID).
+struct SwigluCall {
+  int nE, I;
+  int64_t R;
+  const void* Xp;
+  const int32_t* counts;
+  const int32_t* offsets;
+  const void* W13p;
+  const void* W2;
+  const float* row_scale;
+  int scale_kind;
+  void* AB;   // forward: out (NULL = keep nothing for a backward pass); backward: in
+  void* H;    // forward: out; backward: in
+  void* Yp;   // forward: out, float
+  const void* dYp;
+  void* dAB;
+  void* dXp;
+  void* dW13p;
+  void* dW2;
+  float* qpart;  // backward: [swiglu_qparts][R] partial row dots <dH_r, H_r>, or NULL
+  int accumulate;
+  int32_t* status;
+  // gather-fused dispatch (both or neither): rows of the permuted operand are fetched from X inside the kernels
+  const void* X;
+  const int32_t* slot_of_row;
+};
+
 template <typename T>
-int simt_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
-                    const int32_t* offsets, const void* W13p, const void* W2, void* AB, void* H, void* Yp,
-                    cudaStream_t s);
+int simt_swiglu_fwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s);
 template <typename T>
-int simt_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
-                    const int32_t* offsets, const void* W13p, const void* W2, const void* AB, const void* H,
-                    const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, cudaStream_t s);
+int simt_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s);
 
 // Tensor-core (tcgen05) path, bf16 only.
 enum { TC_ROWS = 0, TC_WGRAD = 1 };
 enum { TC_EPI_SWIGLU_FWD = 0, TC_EPI_F32 = 1, TC_EPI_SWIGLU_BWD = 2, TC_EPI_WGRAD_BF16 = 3, TC_EPI_T_F32 = 4 };
 bool tc_supported(const c2r_config* cfg, int nE, int I, int64_t R);
-// X / slot_of_row (both or neither): the rows of the permuted operand are fetched from X inside the kernels
-// (TMA row gather) and Xp is not read.
-int tc_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
-                  const int32_t* offsets, const void* W13p, const void* W2, void* AB, void* H, void* Yp,
-                  int32_t* status, cudaStream_t s, const void* X = nullptr, const int32_t* slot_of_row = nullptr);
-int tc_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
-                  const int32_t* offsets, const void* W13p, const void* W2, const void* AB, const void* H,
-                  const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status,
-                  cudaStream_t s, const void* X = nullptr, const int32_t* slot_of_row = nullptr);
+int tc_swiglu_fwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s);
+int tc_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s);
+// Rows of the partial-dot buffer the backward call writes for this shape (depends on which kernel serves it).
+int swiglu_qparts(const c2r_config* cfg, int nE, int I, int64_t R);
 
 // Gate logits on the tensor cores (bf16 only).
 bool gate_tc_supported(const c2r_config* cfg);
@@ -64,7 +89,17 @@ int gate_logits_impl(const c2r_config* cfg, const void* X, const void* Wg, const
 int tc_gate_wgrad(const c2r_config* cfg, const void* X, const void* dLd, float* partial, int n_splits,
                   const int32_t* split_counts, const int32_t* split_offsets, int32_t* status, cudaStream_t s);
 
+// c2r_route that can also leave the dispatch's per-block expert histogram in block_counts (may be NULL).
+int route_impl(const c2r_config* cfg, const float* L, const uint64_t* mask, int32_t* idx, float* w, float* p,
+               int32_t* status, int32_t* block_counts, void* stream);
+// c2r_permute with its options: have_hist = block_counts (the workspace) already holds the histogram route_impl
+// wrote; w / w_row: also write the routing weight of every permuted row.
+int permute_call(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X, int32_t* counts,
+                 int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp, int32_t* status, void* ws,
+                 size_t ws_bytes, void* stream, bool have_hist, const float* w, float* w_row);
+
 size_t permute_ws_bytes(const c2r_config* cfg);
+size_t layer_ws_bytes(const c2r_config* cfg);
 size_t gate_bwd_ws_bytes(const c2r_config* cfg);
 size_t dispatch_dedup_ws_bytes(const c2r_config* cfg);
 

@@ -50,6 +50,7 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(SimtGemm g) {
   __shared__ float sa[SK][ST + 4];
   __shared__ float sb[SK][ST + 4];
   __shared__ float sb2[SK][ST + 4];  // up-projection tile of the fused SwiGLU forward
+  __shared__ float sred[ST][17];     // per-row partial dots of the SwiGLU backward, one column per thread column
   const bool dual = g.epi == SIMT_EPI_SWIGLU_FWD;
   const int grp = blockIdx.z;
   int M, Kd;
@@ -116,10 +117,18 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(SimtGemm g) {
     __syncthreads();
   }
   TC* C = (TC*)g.C + c_off;
+  const bool want_q = g.epi == SIMT_EPI_SWIGLU_BWD && g.qpart != nullptr;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int m = m0 + ty * 4 + i;
+    float qrow = 0.f;
+    if (want_q) sred[ty * 4 + i][tx] = 0.f;
     if (m >= M) continue;
+    float sc = 1.f;  // per-row scale of H (SwiGLU forms)
+    if (g.scale_kind != 0 && g.row_scale != nullptr) {
+      const float v = g.row_scale[r0 + m];
+      sc = g.scale_kind == 2 ? 1.0f / (1.0f + expf(-v)) : v;
+    }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int n = n0 + tx * 4 + j;
@@ -141,14 +150,25 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(SimtGemm g) {
           sv[pg] = from_f32<T>(b * (sg + as - as * sg));
           sv[pu] = from_f32<T>(as);
         }
-        ((T*)g.aux_out)[(long long)(r0 + m) * g.I + n] = from_f32<T>(as * b);
+        ((T*)g.aux_out)[(long long)(r0 + m) * g.I + n] = from_f32<T>(sc * (as * b));
       } else {  // SIMT_EPI_SWIGLU_BWD: v = dH[r, n]; dA = dH * (dH/dA), dB = dH * (dH/dB) at the packed columns
         const int pg = pack_col(n, g.I), pu = pg + pack_width(n, g.I);
         const T* sv = (const T*)g.aux + (long long)(r0 + m) * 2 * g.I;
         T* dab = (T*)g.C + (long long)(r0 + m) * 2 * g.I;
-        dab[pg] = from_f32<T>(v * to_f32(sv[pg]));
-        dab[pu] = from_f32<T>(v * to_f32(sv[pu]));
+        dab[pg] = from_f32<T>(sc * v * to_f32(sv[pg]));
+        dab[pu] = from_f32<T>(sc * v * to_f32(sv[pu]));
+        if (want_q) qrow = fmaf(v, to_f32(((const T*)g.aux2)[(long long)(r0 + m) * g.I + n]), qrow);
       }
+    }
+    if (want_q) sred[ty * 4 + i][tx] = qrow;
+  }
+  if (want_q) {  // (uniform across the block) row dots <dH_r, H_r> over this block's 64 columns, in column order
+    __syncthreads();
+    if (tid < ST && m0 + tid < M) {
+      float q = 0.f;
+#pragma unroll
+      for (int x = 0; x < 16; ++x) q += sred[tid][x];
+      g.qpart[(long long)blockIdx.x * g.R + r0 + m0 + tid] = q;
     }
   }
 }
@@ -163,69 +183,60 @@ int simt_launch(const SimtGemm& g, int n_groups, int max_m, cudaStream_t s) {
 }
 
 template <typename T>
-int simt_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
-                    const int32_t* offsets, const void* W13p, const void* W2, void* AB, void* H, void* Yp,
-                    cudaStream_t s) {
-  const int d = cfg->d;
-  const int max_m = (int)R;
+int simt_swiglu_fwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
+  const int d = cfg->d, I = a.I;
+  const int max_m = (int)a.R;
   SimtGemm g{};
-  g.counts = counts; g.offsets = offsets; g.mode = SIMT_ROWS; g.I = I;
-  // A = Xp W1^T, B = Xp W3^T in one pass over Xp; epilogue stores H = silu(A) * B and its two local derivatives
-  g.epi = SIMT_EPI_SWIGLU_FWD; g.aux_out = H;
-  g.A = Xp; g.sam = d; g.sak = 1; g.B = W13p; g.sbn = d; g.sbk = 1; g.sB = (long long)2 * I * d;
-  g.C = AB; g.ldc = 2 * I; g.Ndim = I; g.Kdim = d;
-  int rc = simt_launch<T>(g, nE, max_m, s);
+  g.counts = a.counts; g.offsets = a.offsets; g.mode = SIMT_ROWS; g.I = I; g.R = a.R;
+  // A = Xp W1^T, B = Xp W3^T in one pass over Xp; epilogue stores H = s silu(A) * B and the two local derivatives
+  g.epi = SIMT_EPI_SWIGLU_FWD; g.aux_out = a.H;
+  g.row_scale = a.row_scale; g.scale_kind = a.row_scale ? a.scale_kind : 0;
+  g.A = a.Xp; g.sam = d; g.sak = 1; g.B = a.W13p; g.sbn = d; g.sbk = 1; g.sB = (long long)2 * I * d;
+  g.C = a.AB; g.ldc = 2 * I; g.Ndim = I; g.Kdim = d;
+  int rc = simt_launch<T>(g, a.nE, max_m, s);
   if (rc) return rc;
-  g.epi = SIMT_EPI_STORE; g.aux_out = nullptr;
+  g.epi = SIMT_EPI_STORE; g.aux_out = nullptr; g.row_scale = nullptr; g.scale_kind = 0;
   // Yp = H W2^T  (fp32 partial result)
-  g.A = H; g.sam = I; g.sak = 1; g.B = W2; g.sbn = I; g.sbk = 1; g.sB = (long long)d * I;
-  g.C = Yp; g.ldc = d; g.Ndim = d; g.Kdim = I;
-  return simt_launch<T, float>(g, nE, max_m, s);
+  g.A = a.H; g.sam = I; g.sak = 1; g.B = a.W2; g.sbn = I; g.sbk = 1; g.sB = (long long)d * I;
+  g.C = a.Yp; g.ldc = d; g.Ndim = d; g.Kdim = I;
+  return simt_launch<T, float>(g, a.nE, max_m, s);
 }
 
 template <typename T>
-int simt_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
-                    const int32_t* offsets, const void* W13p, const void* W2, const void* AB, const void* H,
-                    const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, cudaStream_t s) {
-  const int d = cfg->d;
-  const int max_m = (int)R;
+int simt_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
+  const int d = cfg->d, I = a.I, nE = a.nE;
+  const int max_m = (int)a.R;
   SimtGemm g{};
-  g.counts = counts; g.offsets = offsets; g.I = I;
-  // dH = dYp W2  (epilogue turns it into dA, dB at the packed columns)
-  g.mode = SIMT_ROWS; g.epi = SIMT_EPI_SWIGLU_BWD; g.aux = AB;
-  g.A = dYp; g.sam = d; g.sak = 1; g.B = W2; g.sbn = 1; g.sbk = I; g.sB = (long long)d * I;
-  g.C = dAB; g.ldc = 2 * I; g.Ndim = I; g.Kdim = d;
+  g.counts = a.counts; g.offsets = a.offsets; g.I = I; g.R = a.R;
+  // dH = dYp W2  (epilogue turns it into dA, dB at the packed columns, and the row dots with H)
+  g.mode = SIMT_ROWS; g.epi = SIMT_EPI_SWIGLU_BWD; g.aux = a.AB; g.aux2 = a.H; g.qpart = a.qpart;
+  g.row_scale = a.row_scale; g.scale_kind = a.row_scale ? a.scale_kind : 0;
+  g.A = a.dYp; g.sam = d; g.sak = 1; g.B = a.W2; g.sbn = 1; g.sbk = I; g.sB = (long long)d * I;
+  g.C = a.dAB; g.ldc = 2 * I; g.Ndim = I; g.Kdim = d;
   int rc = simt_launch<T>(g, nE, max_m, s);
   if (rc) return rc;
   // dXp = dAB W13p  (fp32 partial result)
-  g.epi = SIMT_EPI_STORE; g.aux = nullptr;
-  g.A = dAB; g.sam = 2 * I; g.sak = 1; g.B = W13p; g.sbn = 1; g.sbk = d; g.sB = (long long)2 * I * d;
-  g.C = dXp; g.ldc = d; g.Ndim = d; g.Kdim = 2 * I;
+  g.epi = SIMT_EPI_STORE; g.aux = nullptr; g.aux2 = nullptr; g.qpart = nullptr; g.row_scale = nullptr; g.scale_kind = 0;
+  g.A = a.dAB; g.sam = 2 * I; g.sak = 1; g.B = a.W13p; g.sbn = 1; g.sbk = d; g.sB = (long long)2 * I * d;
+  g.C = a.dXp; g.ldc = d; g.Ndim = d; g.Kdim = 2 * I;
   rc = simt_launch<T, float>(g, nE, max_m, s);
   if (rc) return rc;
   // dW2_e = dYp_e^T H_e   [d, I]
-  g.mode = SIMT_WGRAD; g.accumulate = accumulate;
-  g.A = dYp; g.sam = 1; g.sak = d; g.B = H; g.sbn = 1; g.sbk = I;
-  g.C = dW2; g.ldc = I; g.sC = (long long)d * I; g.Mdim = d; g.Ndim = I;
+  g.mode = SIMT_WGRAD; g.accumulate = a.accumulate;
+  g.A = a.dYp; g.sam = 1; g.sak = d; g.B = a.H; g.sbn = 1; g.sbk = I;
+  g.C = a.dW2; g.ldc = I; g.sC = (long long)d * I; g.Mdim = d; g.Ndim = I;
   rc = simt_launch<T>(g, nE, d, s);
   if (rc) return rc;
   // dW13p_e = dAB_e^T Xp_e   [2I, d]
-  g.A = dAB; g.sam = 1; g.sak = 2 * I; g.B = Xp; g.sbn = 1; g.sbk = d;
-  g.C = dW13p; g.ldc = d; g.sC = (long long)2 * I * d; g.Mdim = 2 * I; g.Ndim = d;
+  g.A = a.dAB; g.sam = 1; g.sak = 2 * I; g.B = a.Xp; g.sbn = 1; g.sbk = d;
+  g.C = a.dW13p; g.ldc = d; g.sC = (long long)2 * I * d; g.Mdim = 2 * I; g.Ndim = d;
   return simt_launch<T>(g, nE, 2 * I, s);
 }
 
-template int simt_swiglu_fwd<float>(const c2r_config*, int, int, int64_t, const void*, const int32_t*, const int32_t*,
-                                    const void*, const void*, void*, void*, void*, cudaStream_t);
-template int simt_swiglu_fwd<__nv_bfloat16>(const c2r_config*, int, int, int64_t, const void*, const int32_t*,
-                                            const int32_t*, const void*, const void*, void*, void*, void*,
-                                            cudaStream_t);
-template int simt_swiglu_bwd<float>(const c2r_config*, int, int, int64_t, const void*, const int32_t*, const int32_t*,
-                                    const void*, const void*, const void*, const void*, const void*, void*, void*,
-                                    void*, void*, int, cudaStream_t);
-template int simt_swiglu_bwd<__nv_bfloat16>(const c2r_config*, int, int, int64_t, const void*, const int32_t*,
-                                            const int32_t*, const void*, const void*, const void*, const void*,
-                                            const void*, void*, void*, void*, void*, int, cudaStream_t);
+template int simt_swiglu_fwd<float>(const c2r_config*, const SwigluCall&, cudaStream_t);
+template int simt_swiglu_fwd<__nv_bfloat16>(const c2r_config*, const SwigluCall&, cudaStream_t);
+template int simt_swiglu_bwd<float>(const c2r_config*, const SwigluCall&, cudaStream_t);
+template int simt_swiglu_bwd<__nv_bfloat16>(const c2r_config*, const SwigluCall&, cudaStream_t);
 
 }  // namespace c2r
 

@@ -49,9 +49,13 @@ struct TcParams {
   const int32_t* counts;
   const int32_t* offsets;
   void* C;         // main output
-  const void* AB;  // TC_EPI_SWIGLU_BWD: saved (A, B)
-  void* H;         // TC_EPI_SWIGLU_FWD: H output
+  const void* AB;  // TC_EPI_SWIGLU_BWD: the two local derivatives the forward pass saved
+  void* H;         // TC_EPI_SWIGLU_FWD: H output; TC_EPI_SWIGLU_BWD: the forward's H (read for the row dots), may be NULL
   int32_t* status;
+  // per-row scale of H (SwiGLU forms): H = s_r silu(A) B, s_r = row_scale[r] (kind 1) or sigmoid(row_scale[r]) (kind 2)
+  const float* row_scale;
+  int scale_kind;
+  float* qpart;    // TC_EPI_SWIGLU_BWD: [2 * n_tiles][R] partial row dots <dH_r, H_r>, or NULL
   // row-gathering variants: the operand's rows are token rows of X picked through slot_of_row
   const int32_t* slot_of_row;  // [R], -1 = padding (reads zeros)
   int slots_per_token;         // K of the routing
@@ -192,6 +196,14 @@ __device__ __forceinline__ int4 gather_rows(const TcParams& p, int r) {
   if (r >= 0 && r + 3 < p.R) s = *reinterpret_cast<const int4*>(p.slot_of_row + r);
   const int K = p.slots_per_token, oob = p.n_tokens;
   return make_int4(s.x < 0 ? oob : s.x / K, s.y < 0 ? oob : s.y / K, s.z < 0 ? oob : s.z / K, s.w < 0 ? oob : s.w / K);
+}
+
+// Scale of row r (see TcParams::row_scale); rows that do not exist get 0.
+__device__ __forceinline__ float row_scale_of(const TcParams& p, long long r, bool valid) {
+  if (p.scale_kind == 0 || p.row_scale == nullptr) return 1.f;
+  if (!valid) return 0.f;
+  const float v = p.row_scale[r];
+  return p.scale_kind == 2 ? 1.0f / (1.0f + expf(-v)) : v;
 }
 
 // A_MN / B_MN: operand is MN-major in global memory (the contraction index is the row index).
@@ -412,11 +424,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const int rows_valid = max(0, min(32, ti.m_end - row0));
       const long long mrow = row0 + lane;
       bool waited = !have_acc;
+      const float sc = row_scale_of(p, mrow, lane < rows_valid);  // requested before the accumulator is awaited
       if (p.epi == TC_EPI_SWIGLU_BWD) {
-        // dA = dH * (dH/dA), dB = dH * (dH/dB) on groups of 64 H columns; the forward pass saved both
-        // local derivatives.  They do not depend on the accumulator, so the first group's loads are
-        // issued before it is awaited.
+        // dA = s_r dH (dH/dA), dB = s_r dH (dH/dB) on groups of 64 H columns, s_r the row's scale; the forward pass
+        // saved both local derivatives.  With qpart, also the row dot <dH_r, H_r> over this warp's columns (H as the
+        // forward stored it, scale included): the gradient w.r.t. the scale times the scale.  None of the loads
+        // depends on the accumulator, so the first group's are issued before it is awaited.
         const int n_groups = (w + 63) >> 6;
+        const bool want_q = p.qpart != nullptr;
+        float qacc = 0.f;
         for (int g = hsel; g < n_groups; g += 2) {
           const int hc0 = TILE_N * ti.jn + 64 * g;  // first H column of the group; a group never leaves its
           const int blk = hc0 >> 7;                 // 128-channel block of the packed (A | B) layout
@@ -426,17 +442,41 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const long long pitch = 4ll * p.I;  // bytes per row of AB / dAB
           const uint8_t* gsrc = (const uint8_t*)p.AB + row0 * pitch;
           uint8_t* go = (uint8_t*)p.C + row0 * pitch;
-          uint4 in0[8], in1[8];  // both pieces are requested before either is parked in shared memory
+          // Loads are requested ahead of their use, but staged one piece at a time so that at most two pieces
+          // (64 registers) are in flight per thread.
+          uint4 in0[8], in1[8];
+          if (want_q) {  // the H piece, for the row dots
+            global_rows_load(in1, (const uint8_t*)p.H + row0 * (2ll * p.I) + 2 * hc0, 2ll * p.I, rows_valid, vbytes, lane);
+            stage_rows_store(buf1, in1, lane);
+          }
           global_rows_load(in0, gsrc + 2 * col_a, pitch, rows_valid, vbytes, lane);
           global_rows_load(in1, gsrc + 2 * col_b, pitch, rows_valid, vbytes, lane);
           stage_rows_store(buf0, in0, lane);
-          stage_rows_store(buf1, in1, lane);
           __syncwarp();
           if (!waited) {
             if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             waited = true;
           }
+          if (want_q) {
+            // pass 1 over the accumulator columns of the group: q += <dH_r, H_r>
+#pragma unroll
+            for (int pc = 0; pc < 4; ++pc) {
+              if (32 * pc >= vbytes) break;  // warp-uniform
+              uint32_t r0[16];
+              float hv[16];
+              if (have_acc) {
+                tc_ld16(taddr_row + 64 * g + 16 * pc, r0);
+                tc_ld_wait();
+              }
+              unpack_bf16x16(lds128(stg_addr(buf1, lane, 2 * pc)), lds128(stg_addr(buf1, lane, 2 * pc + 1)), hv);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) qacc = fmaf(have_acc ? __uint_as_float(r0[i]) : 0.f, hv[i], qacc);
+            }
+            __syncwarp();
+          }
+          stage_rows_store(buf1, in1, lane);
+          __syncwarp();
 #pragma unroll
           for (int pc = 0; pc < 4; ++pc) {
             if (32 * pc >= vbytes) break;  // warp-uniform
@@ -447,7 +487,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               tc_ld_wait();
             }
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v0[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
+            for (int i = 0; i < 16; ++i) v0[i] = have_acc ? sc * __uint_as_float(r0[i]) : 0.f;
             const uint32_t sa0 = stg_addr(buf0, lane, 2 * pc), sa1 = stg_addr(buf0, lane, 2 * pc + 1);
             const uint32_t sb0 = stg_addr(buf1, lane, 2 * pc), sb1 = stg_addr(buf1, lane, 2 * pc + 1);
             unpack_bf16x16(lds128(sa0), lds128(sa1), ga);
@@ -463,6 +503,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           __syncwarp();
         }
         if (!ok) break;
+        // one partial per (row, N tile, warp of the lane quarter); a warp without a group writes its zero
+        if (want_q && lane < rows_valid) p.qpart[(long long)(2 * ti.jn + hsel) * p.R + mrow] = qacc;
       }
       if (!waited) {
         if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
@@ -493,7 +535,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               const float b = have_acc ? __uint_as_float(r1[i]) : 0.f;
               const float sg = sigmoid_fast(a);
               const float as = a * sg;             // silu(a)
-              h[i] = as * b;
+              h[i] = sc * (as * b);
               ga[i] = b * (sg + as - as * sg);     // b silu'(a), silu'(a) = s (1 + a (1 - s))
               gb[i] = as;
             }
@@ -664,76 +706,81 @@ bool tc_supported(const c2r_config* cfg, int nE, int I, int64_t R) {
          (nE == 1 || cfg->row_align % BM == 0) && get_encode() != nullptr;
 }
 
-int tc_swiglu_fwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
-                  const int32_t* offsets, const void* W13p, const void* W2, void* AB, void* H, void* Yp,
-                  int32_t* status, cudaStream_t s, const void* X, const int32_t* slot_of_row) {
-  const int d = cfg->d;
+int swiglu_qparts(const c2r_config* cfg, int nE, int I, int64_t R) {
+  return tc_supported(cfg, nE, I, R) ? 2 * ((I + TILE_N - 1) / TILE_N) : (I + 63) / 64;
+}
+
+int tc_swiglu_fwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
+  const int d = cfg->d, I = a.I, nE = a.nE;
+  const int64_t R = a.R;
   CUtensorMap ma, mb;
   TcParams p{};
-  p.mode = TC_ROWS; p.n_experts = nE; p.R = (int)R; p.I = I; p.counts = counts; p.offsets = offsets; p.status = status;
+  p.mode = TC_ROWS; p.n_experts = nE; p.R = (int)R; p.I = I; p.counts = a.counts; p.offsets = a.offsets; p.status = a.status;
   // (A | B) = Xp W13p^T with the SwiGLU epilogue: AB packed + H
-  const bool gather = X != nullptr && slot_of_row != nullptr;  // rows of X picked inside the GEMM, no permuted copy
-  int rc = gather ? make_map(&ma, X, d, cfg->N, 0, BK, 1) : make_map(&ma, Xp, d, R, 0, BK, BM);
+  const bool gather = a.X != nullptr && a.slot_of_row != nullptr;  // rows of X picked inside the GEMM, no permuted copy
+  int rc = gather ? make_map(&ma, a.X, d, cfg->N, 0, BK, 1) : make_map(&ma, a.Xp, d, R, 0, BK, BM);
   if (rc) return rc;
-  rc = make_map(&mb, W13p, d, 2 * I, nE, BK, 128);
+  rc = make_map(&mb, a.W13p, d, 2 * I, nE, BK, 128);
   if (rc) return rc;
-  p.epi = TC_EPI_SWIGLU_FWD; p.K = d; p.Nout = I; p.n_tiles = (I + 127) / 128; p.C = AB; p.H = H;
-  p.slot_of_row = slot_of_row; p.slots_per_token = cfg->K; p.n_tokens = cfg->N;
+  p.epi = TC_EPI_SWIGLU_FWD; p.K = d; p.Nout = I; p.n_tiles = (I + 127) / 128; p.C = a.AB; p.H = a.H;
+  p.row_scale = a.row_scale; p.scale_kind = a.row_scale ? a.scale_kind : 0;
+  p.slot_of_row = a.slot_of_row; p.slots_per_token = cfg->K; p.n_tokens = cfg->N;
   rc = gather ? launch<false, false, 1>(ma, mb, p, s) : launch<false, false>(ma, mb, p, s);
   if (rc) return rc;
   // Yp = H W2^T (fp32)
-  rc = make_map(&ma, H, I, R, 0, BK, BM);
+  rc = make_map(&ma, a.H, I, R, 0, BK, BM);
   if (rc) return rc;
-  rc = make_map(&mb, W2, I, d, nE, BK, 128);
+  rc = make_map(&mb, a.W2, I, d, nE, BK, 128);
   if (rc) return rc;
-  p.epi = TC_EPI_F32; p.K = I; p.Nout = d; p.n_tiles = (d + TILE_N - 1) / TILE_N; p.C = Yp; p.ldc = d; p.H = nullptr;
+  p.epi = TC_EPI_F32; p.K = I; p.Nout = d; p.n_tiles = (d + TILE_N - 1) / TILE_N; p.C = a.Yp; p.ldc = d; p.H = nullptr;
+  p.row_scale = nullptr; p.scale_kind = 0;
   return launch<false, false>(ma, mb, p, s);
 }
 
-int tc_swiglu_bwd(const c2r_config* cfg, int nE, int I, int64_t R, const void* Xp, const int32_t* counts,
-                  const int32_t* offsets, const void* W13p, const void* W2, const void* AB, const void* H,
-                  const void* dYp, void* dAB, void* dXp, void* dW13p, void* dW2, int accumulate, int32_t* status,
-                  cudaStream_t s, const void* X, const int32_t* slot_of_row) {
-  const int d = cfg->d;
+int tc_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
+  const int d = cfg->d, I = a.I, nE = a.nE;
+  const int64_t R = a.R;
   CUtensorMap ma, mb;
   TcParams p{};
-  p.n_experts = nE; p.R = (int)R; p.I = I; p.counts = counts; p.offsets = offsets; p.status = status;
+  p.n_experts = nE; p.R = (int)R; p.I = I; p.counts = a.counts; p.offsets = a.offsets; p.status = a.status;
   // dH = dYp W2 -> (dA | dB) packed
   p.mode = TC_ROWS;
-  int rc = make_map(&ma, dYp, d, R, 0, BK, BM);
+  int rc = make_map(&ma, a.dYp, d, R, 0, BK, BM);
   if (rc) return rc;
-  rc = make_map(&mb, W2, I, d, nE, 64, 64);  // W2_e is [d (k)][I (n)]: MN-major B
+  rc = make_map(&mb, a.W2, I, d, nE, 64, 64);  // W2_e is [d (k)][I (n)]: MN-major B
   if (rc) return rc;
-  p.epi = TC_EPI_SWIGLU_BWD; p.K = d; p.Nout = I; p.n_tiles = (I + TILE_N - 1) / TILE_N; p.C = dAB; p.AB = AB;
+  p.epi = TC_EPI_SWIGLU_BWD; p.K = d; p.Nout = I; p.n_tiles = (I + TILE_N - 1) / TILE_N; p.C = a.dAB; p.AB = a.AB;
+  p.row_scale = a.row_scale; p.scale_kind = a.row_scale ? a.scale_kind : 0; p.qpart = a.qpart; p.H = a.H;
   rc = launch<false, true>(ma, mb, p, s);
   if (rc) return rc;
+  p.row_scale = nullptr; p.scale_kind = 0; p.qpart = nullptr; p.H = nullptr;
   // dXp = dAB W13p (fp32)
-  rc = make_map(&ma, dAB, 2 * I, R, 0, BK, BM);
+  rc = make_map(&ma, a.dAB, 2 * I, R, 0, BK, BM);
   if (rc) return rc;
-  rc = make_map(&mb, W13p, d, 2 * I, nE, 64, 64);  // W13p_e is [2I (k)][d (n)]: MN-major B
+  rc = make_map(&mb, a.W13p, d, 2 * I, nE, 64, 64);  // W13p_e is [2I (k)][d (n)]: MN-major B
   if (rc) return rc;
-  p.epi = TC_EPI_F32; p.K = 2 * I; p.Nout = d; p.n_tiles = (d + TILE_N - 1) / TILE_N; p.C = dXp; p.ldc = d; p.AB = nullptr;
+  p.epi = TC_EPI_F32; p.K = 2 * I; p.Nout = d; p.n_tiles = (d + TILE_N - 1) / TILE_N; p.C = a.dXp; p.ldc = d; p.AB = nullptr;
   rc = launch<false, true>(ma, mb, p, s);
   if (rc) return rc;
   // dW2_e = dYp_e^T H_e  [d, I]
-  p.mode = TC_WGRAD; p.epi = TC_EPI_WGRAD_BF16; p.accumulate = accumulate;
-  rc = make_map(&ma, dYp, d, R, 0, 64, 64);
+  p.mode = TC_WGRAD; p.epi = TC_EPI_WGRAD_BF16; p.accumulate = a.accumulate;
+  rc = make_map(&ma, a.dYp, d, R, 0, 64, 64);
   if (rc) return rc;
-  rc = make_map(&mb, H, I, R, 0, 64, 64);
+  rc = make_map(&mb, a.H, I, R, 0, 64, 64);
   if (rc) return rc;
   p.Mout = d; p.Nout = I; p.m_tiles = (d + TILE_M - 1) / TILE_M; p.n_tiles = (I + TILE_N - 1) / TILE_N;
-  p.C = dW2; p.ldc = I; p.sC = (long long)d * I;
+  p.C = a.dW2; p.ldc = I; p.sC = (long long)d * I;
   rc = launch<true, true>(ma, mb, p, s);
   if (rc) return rc;
   // dW13p_e = dAB_e^T Xp_e  [2I, d]
-  rc = make_map(&ma, dAB, 2 * I, R, 0, 64, 64);
+  rc = make_map(&ma, a.dAB, 2 * I, R, 0, 64, 64);
   if (rc) return rc;
-  const bool gather = X != nullptr && slot_of_row != nullptr;
-  rc = gather ? make_map(&mb, X, d, cfg->N, 0, 64, 1) : make_map(&mb, Xp, d, R, 0, 64, 64);
+  const bool gather = a.X != nullptr && a.slot_of_row != nullptr;
+  rc = gather ? make_map(&mb, a.X, d, cfg->N, 0, 64, 1) : make_map(&mb, a.Xp, d, R, 0, 64, 64);
   if (rc) return rc;
   p.Mout = 2 * I; p.Nout = d; p.m_tiles = (2 * I + TILE_M - 1) / TILE_M; p.n_tiles = (d + TILE_N - 1) / TILE_N;
-  p.C = dW13p; p.ldc = d; p.sC = (long long)2 * I * d;
-  p.slot_of_row = slot_of_row; p.slots_per_token = cfg->K; p.n_tokens = cfg->N;
+  p.C = a.dW13p; p.ldc = d; p.sC = (long long)2 * I * d;
+  p.slot_of_row = a.slot_of_row; p.slots_per_token = cfg->K; p.n_tokens = cfg->N;
   return gather ? launch<true, true, 2>(ma, mb, p, s) : launch<true, true>(ma, mb, p, s);
 }
 

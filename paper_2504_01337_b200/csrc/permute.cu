@@ -5,9 +5,10 @@
 
 namespace c2r {
 
-constexpr int PERM_WARPS = 8;                 // warps per block
-constexpr int PERM_ITERS = 2;                 // 32-slot iterations per warp
-constexpr int PERM_BLOCK_SLOTS = PERM_WARPS * PERM_ITERS * 32;
+// Blocking of the counting sort: a block owns perm_tokens_per_block(K) consecutive tokens, i.e. at most 512
+// consecutive slots, a whole number of 32-slot groups.  One warp per group.
+constexpr int PERM_THREADS = 512;
+constexpr int PERM_GROUPS = PERM_THREADS / 32;  // 32-slot groups a block can own
 
 __device__ __forceinline__ uint32_t lanemask_lt() {
   uint32_t m;
@@ -15,43 +16,66 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
   return m;
 }
 
-// Per-warp, per-expert counts of this block's slots.  A warp owns PERM_ITERS*32 consecutive
-// slots; inside a 32-slot group, lanes with equal expert form a peer set (match.any) whose
-// lowest lane adds the set size -- no atomics, and the order of slots is preserved.
-// skip_negative: a key of -1 marks a slot that takes no part (used by the de-duplicated dispatch).
-__device__ __forceinline__ void warp_count(const int32_t* __restrict__ idx, long long NK, int E, int (*warp_cnt)[64],
-                                           int e_reg[PERM_ITERS], int& flags, int skip_negative) {
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const long long base = (long long)blockIdx.x * PERM_BLOCK_SLOTS + (long long)w * PERM_ITERS * 32;
-#pragma unroll
-  for (int it = 0; it < PERM_ITERS; ++it) {
-    const long long s = base + it * 32 + lane;
-    int e = -1;
-    if (s < NK) {
-      e = idx[s];
-      if ((e < 0 || e >= E) && !(skip_negative && e == -1)) { flags |= C2R_STATUS_BAD_INDEX; e = min(max(e, 0), E - 1); }
-    }
-    e_reg[it] = e;
-    const uint32_t peers = __match_any_sync(0xffffffffu, e);
-    if (e >= 0 && lane == __ffs(peers) - 1) warp_cnt[w][e] += __popc(peers);
-    __syncwarp();
+// Expert key of slot s (clamped into [0,E); -1 = the slot takes no part: past the end, or a key of -1 when
+// skip_negative is set, which the de-duplicated dispatch uses).
+__device__ __forceinline__ int slot_key(const int32_t* __restrict__ idx, long long s, long long NK, int E, int skip_negative,
+                                        int& flags) {
+  if (s >= NK) return -1;
+  int e = idx[s];
+  if (e < 0 || e >= E) {
+    if (skip_negative && e == -1) return -1;
+    flags |= C2R_STATUS_BAD_INDEX;
+    e = min(max(e, 0), E - 1);
   }
+  return e;
 }
 
-__global__ void __launch_bounds__(PERM_WARPS * 32) perm_hist_kernel(const int32_t* __restrict__ idx, long long NK, int E,
-                                                                    int32_t* __restrict__ block_counts,
-                                                                    int32_t* __restrict__ status, int skip_negative) {
-  __shared__ int warp_cnt[PERM_WARPS][64];
-  for (int i = threadIdx.x; i < PERM_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
+// Per-group, per-expert counts of this block's slots: inside a 32-slot group, lanes with equal expert form a
+// peer set (match.any) whose lowest lane records the set size -- no atomics, and the order of slots is kept.
+// grp_cnt must be zero on entry.  Returns this thread's key.
+__device__ __forceinline__ int group_count(const int32_t* __restrict__ idx, long long NK, int E, int slots_per_block,
+                                           int (*grp_cnt)[64], int& flags, int skip_negative) {
+  const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
+  int e = -1;
+  if (32 * g < slots_per_block)
+    e = slot_key(idx, (long long)blockIdx.x * slots_per_block + threadIdx.x, NK, E, skip_negative, flags);
+  const uint32_t peers = __match_any_sync(0xffffffffu, e);
+  if (e >= 0 && lane == __ffs(peers) - 1) grp_cnt[g][e] = __popc(peers);
+  return e;
+}
+
+// Layout position -> expert from expert_rank (NULL = identity).  A table that is not a permutation of
+// [0,E) (an entry out of range, a duplicate, hence a hole) is replaced by the identity order and reported.
+// All threads of the block must call; needs E <= 64 <= blockDim.x.  Ends with a barrier.
+__device__ __forceinline__ void layout_order(const int32_t* __restrict__ expert_rank, int E, int* s_by_rank, int* s_bad) {
+  if (threadIdx.x < 64) s_by_rank[threadIdx.x] = -1;
+  if (threadIdx.x == 0) *s_bad = 0;
   __syncthreads();
-  int e_reg[PERM_ITERS];
+  if ((int)threadIdx.x < E) {
+    const int r = expert_rank ? expert_rank[threadIdx.x] : (int)threadIdx.x;
+    if (r < 0 || r >= E) *s_bad = 1;
+    else s_by_rank[r] = threadIdx.x;  // duplicates: one writer wins and some other position stays -1
+  }
+  __syncthreads();
+  if ((int)threadIdx.x < E && s_by_rank[threadIdx.x] < 0) *s_bad = 1;
+  __syncthreads();
+  if (*s_bad && (int)threadIdx.x < E) s_by_rank[threadIdx.x] = threadIdx.x;
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(PERM_THREADS) perm_hist_kernel(const int32_t* __restrict__ idx, long long NK, int E,
+                                                                 int slots_per_block, int32_t* __restrict__ block_counts,
+                                                                 int32_t* __restrict__ status, int skip_negative) {
+  __shared__ int grp_cnt[PERM_GROUPS][64];
+  for (int i = threadIdx.x; i < PERM_GROUPS * 64; i += blockDim.x) (&grp_cnt[0][0])[i] = 0;
+  __syncthreads();
   int flags = 0;
-  warp_count(idx, NK, E, warp_cnt, e_reg, flags, skip_negative);
+  group_count(idx, NK, E, slots_per_block, grp_cnt, flags, skip_negative);
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
     int s = 0;
 #pragma unroll
-    for (int w = 0; w < PERM_WARPS; ++w) s += warp_cnt[w][e];
+    for (int g = 0; g < PERM_GROUPS; ++g) s += grp_cnt[g][e];
     block_counts[(size_t)blockIdx.x * E + e] = s;
   }
   if (status != nullptr && flags) atomicOr(status, flags);
@@ -61,9 +85,11 @@ __global__ void __launch_bounds__(PERM_WARPS * 32) perm_hist_kernel(const int32_
 // 32 blocks per shuffle scan), then the segment offsets in layout (rank) order with alignment.
 __global__ void __launch_bounds__(1024) perm_scan_kernel(int32_t* __restrict__ block_counts, int n_blocks, int E,
                                                          const int32_t* __restrict__ expert_rank, int row_align,
-                                                         int32_t* __restrict__ counts, int32_t* __restrict__ offsets) {
+                                                         int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+                                                         int32_t* __restrict__ status) {
   __shared__ int s_counts[64];
   __shared__ int s_by_rank[64];
+  __shared__ int s_bad;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int e = warp; e < E; e += 32) {
     int running = 0;
@@ -81,12 +107,7 @@ __global__ void __launch_bounds__(1024) perm_scan_kernel(int32_t* __restrict__ b
     }
     if (lane == 0) s_counts[e] = running;
   }
-  if (threadIdx.x < E) {
-    int r = expert_rank ? expert_rank[threadIdx.x] : threadIdx.x;
-    r = min(max(r, 0), E - 1);
-    s_by_rank[r] = threadIdx.x;
-  }
-  __syncthreads();
+  layout_order(expert_rank, E, s_by_rank, &s_bad);
   if (threadIdx.x == 0) {
     int cursor = 0;
     for (int r = 0; r < E; ++r) {
@@ -95,72 +116,84 @@ __global__ void __launch_bounds__(1024) perm_scan_kernel(int32_t* __restrict__ b
       cursor += (s_counts[e] + row_align - 1) / row_align * row_align;
     }
     offsets[E] = cursor;
+    if (s_bad && status != nullptr) atomicOr(status, C2R_STATUS_BAD_INDEX);
   }
   if (threadIdx.x < E) counts[threadIdx.x] = s_counts[threadIdx.x];
 }
 
-// Stable rank of every slot: segment start + slots of the same expert in earlier blocks, earlier
-// warps of this block, earlier 32-groups of this warp, lower lanes of this group.
-__global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_kernel(const int32_t* __restrict__ idx, long long NK, int E,
-                                                                    const int32_t* __restrict__ block_base,
-                                                                    const int32_t* __restrict__ offsets,
-                                                                    int32_t* __restrict__ row_of_slot,
-                                                                    int32_t* __restrict__ slot_of_row, int skip_negative) {
-  __shared__ int warp_cnt[PERM_WARPS][64];
-  for (int i = threadIdx.x; i < PERM_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
-  __syncthreads();
-  int e_reg[PERM_ITERS];
-  int flags = 0;
-  warp_count(idx, NK, E, warp_cnt, e_reg, flags, skip_negative);
-  __syncthreads();
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    int run = offsets[e] + block_base[(size_t)blockIdx.x * E + e];
+// Stable rank of a block's slots once grp_cnt holds the per-group counts and s_start[e] the row at which the
+// block's first slot of expert e lands: rows of earlier groups of the block, then lower lanes of the group.
+// w (optional): w_row[row] = w[slot], the routing weight of the slot that owns the row.
+__device__ __forceinline__ void rank_and_write(int e, long long NK, int E, int slots_per_block, int (*grp_cnt)[64],
+                                               const int* s_start, int32_t* __restrict__ row_of_slot,
+                                               int32_t* __restrict__ slot_of_row, const float* __restrict__ w,
+                                               float* __restrict__ w_row) {
+  for (int x = threadIdx.x; x < E; x += blockDim.x) {
+    int run = s_start[x];
 #pragma unroll
-    for (int w = 0; w < PERM_WARPS; ++w) {
-      const int c = warp_cnt[w][e];
-      warp_cnt[w][e] = run;
+    for (int g = 0; g < PERM_GROUPS; ++g) {
+      const int c = grp_cnt[g][x];
+      grp_cnt[g][x] = run;
       run += c;
     }
   }
   __syncthreads();
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const long long base = (long long)blockIdx.x * PERM_BLOCK_SLOTS + (long long)w * PERM_ITERS * 32;
-#pragma unroll
-  for (int it = 0; it < PERM_ITERS; ++it) {
-    const long long s = base + it * 32 + lane;
-    const int e = e_reg[it];
-    const uint32_t peers = __match_any_sync(0xffffffffu, e);
-    const int start = (e >= 0) ? warp_cnt[w][e] : 0;
-    __syncwarp();
-    if (e >= 0 && lane == __ffs(peers) - 1) warp_cnt[w][e] = start + __popc(peers);
-    __syncwarp();
-    if (e >= 0) {
-      const int row = start + __popc(peers & lanemask_lt());
-      row_of_slot[s] = row;
-      slot_of_row[row] = (int32_t)s;
-    }
+  const int g = threadIdx.x >> 5;
+  const uint32_t peers = __match_any_sync(0xffffffffu, e);
+  if (e >= 0) {
+    const long long s = (long long)blockIdx.x * slots_per_block + threadIdx.x;
+    const int row = grp_cnt[g][e] + __popc(peers & lanemask_lt());
+    row_of_slot[s] = row;
+    slot_of_row[row] = (int32_t)s;
+    if (w_row != nullptr) w_row[row] = w[s];
   }
+}
+
+__global__ void __launch_bounds__(PERM_THREADS) perm_rank_kernel(const int32_t* __restrict__ idx, long long NK, int E,
+                                                                 int slots_per_block,
+                                                                 const int32_t* __restrict__ block_base,
+                                                                 const int32_t* __restrict__ offsets,
+                                                                 int32_t* __restrict__ row_of_slot,
+                                                                 int32_t* __restrict__ slot_of_row, int skip_negative,
+                                                                 const float* __restrict__ w, float* __restrict__ w_row) {
+  __shared__ int grp_cnt[PERM_GROUPS][64];
+  __shared__ int s_start[64];
+  for (int i = threadIdx.x; i < PERM_GROUPS * 64; i += blockDim.x) (&grp_cnt[0][0])[i] = 0;
+  for (int e = threadIdx.x; e < E; e += blockDim.x) s_start[e] = offsets[e] + block_base[(size_t)blockIdx.x * E + e];
+  __syncthreads();
+  int flags = 0;
+  const int e = group_count(idx, NK, E, slots_per_block, grp_cnt, flags, skip_negative);
+  __syncthreads();
+  rank_and_write(e, NK, E, slots_per_block, grp_cnt, s_start, row_of_slot, slot_of_row, w, w_row);
 }
 
 // The scan folded into the rank pass (for batches of at most PERM_FUSED_MAX_BLOCKS blocks): every block
 // adds up the histogram rows of the blocks before it and of all blocks (E columns, coalesced), derives the
-// aligned segment offsets itself, and block 0 publishes counts and offsets.  One launch and one
-// dependent round trip fewer than hist -> scan -> rank.
+// aligned segment offsets itself, and block 0 publishes counts and offsets.  The blocks also mark the rows
+// that hold no slot (the padding that closes every aligned segment and the rows past the layout's end, up
+// to R) with -1 in slot_of_row and 0 in w_row, so the call needs no memset: two launches fewer and one
+// dependent round trip fewer than memset -> hist -> scan -> rank.
 constexpr int PERM_FUSED_MAX_BLOCKS = 1024;
-__global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_fused_kernel(const int32_t* __restrict__ idx, long long NK, int E,
-                                                                          const int32_t* __restrict__ block_counts,
-                                                                          int n_blocks,
-                                                                          const int32_t* __restrict__ expert_rank,
-                                                                          int row_align, int32_t* __restrict__ counts,
-                                                                          int32_t* __restrict__ offsets,
-                                                                          int32_t* __restrict__ row_of_slot,
-                                                                          int32_t* __restrict__ slot_of_row) {
-  __shared__ int warp_cnt[PERM_WARPS][64];
-  __shared__ int s_before[64], s_total[64], s_by_rank[64], s_off[65];
-  __shared__ int s_part[2][PERM_WARPS * 32 / 64][64];  // partial sums: [before | total][quarter of the blocks][expert]
-  for (int i = threadIdx.x; i < PERM_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
+__global__ void __launch_bounds__(PERM_THREADS) perm_rank_fused_kernel(const int32_t* __restrict__ idx, long long NK, int E,
+                                                                       int slots_per_block,
+                                                                       const int32_t* __restrict__ block_counts,
+                                                                       int n_blocks,
+                                                                       const int32_t* __restrict__ expert_rank,
+                                                                       int row_align, long long R,
+                                                                       int32_t* __restrict__ counts,
+                                                                       int32_t* __restrict__ offsets,
+                                                                       int32_t* __restrict__ row_of_slot,
+                                                                       int32_t* __restrict__ slot_of_row,
+                                                                       const float* __restrict__ w,
+                                                                       float* __restrict__ w_row,
+                                                                       int32_t* __restrict__ status) {
+  constexpr int PARTS = PERM_THREADS / 64;
+  __shared__ int grp_cnt[PERM_GROUPS][64];
+  __shared__ int s_start[64], s_total[64], s_by_rank[64], s_off[65];
+  __shared__ int s_part[2][PARTS][64];  // partial sums: [before | total][share of the blocks][expert]
+  __shared__ int s_bad;
+  for (int i = threadIdx.x; i < PERM_GROUPS * 64; i += blockDim.x) (&grp_cnt[0][0])[i] = 0;
   {
-    constexpr int PARTS = PERM_WARPS * 32 / 64;
     const int e = threadIdx.x & 63, part = threadIdx.x >> 6;
     int before = 0, total = 0;
     if (e < E) {
@@ -174,15 +207,13 @@ __global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_fused_kernel(const 
     s_part[0][part][e] = before;
     s_part[1][part][e] = total;
   }
-  __syncthreads();
+  layout_order(expert_rank, E, s_by_rank, &s_bad);  // (its barriers also publish s_part and the zeroed grp_cnt)
   for (int e = threadIdx.x; e < E; e += blockDim.x) {
     int before = 0, total = 0;
 #pragma unroll
-    for (int q = 0; q < PERM_WARPS * 32 / 64; ++q) { before += s_part[0][q][e]; total += s_part[1][q][e]; }
-    s_before[e] = before;
+    for (int q = 0; q < PARTS; ++q) { before += s_part[0][q][e]; total += s_part[1][q][e]; }
+    s_start[e] = before;
     s_total[e] = total;
-    int r = expert_rank ? expert_rank[e] : e;
-    s_by_rank[min(max(r, 0), E - 1)] = e;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -193,10 +224,10 @@ __global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_fused_kernel(const 
       cursor += (s_total[e] + row_align - 1) / row_align * row_align;
     }
     s_off[E] = cursor;
+    if (blockIdx.x == 0 && s_bad && status != nullptr) atomicOr(status, C2R_STATUS_BAD_INDEX);
   }
-  int e_reg[PERM_ITERS];
   int flags = 0;
-  warp_count(idx, NK, E, warp_cnt, e_reg, flags, 0);
+  const int e_mine = group_count(idx, NK, E, slots_per_block, grp_cnt, flags, 0);
   __syncthreads();
   if (blockIdx.x == 0) {
     for (int e = threadIdx.x; e <= E; e += blockDim.x) {
@@ -204,33 +235,23 @@ __global__ void __launch_bounds__(PERM_WARPS * 32) perm_rank_fused_kernel(const 
       if (e < E) counts[e] = s_total[e];
     }
   }
-  for (int e = threadIdx.x; e < E; e += blockDim.x) {
-    int run = s_off[e] + s_before[e];
-#pragma unroll
-    for (int w = 0; w < PERM_WARPS; ++w) {
-      const int c = warp_cnt[w][e];
-      warp_cnt[w][e] = run;
-      run += c;
+  // rows without a slot: expert x's padding is written by block x mod gridDim.x, the tail by the last block
+  for (int x = blockIdx.x; x < E; x += gridDim.x) {
+    const int r0 = s_off[x] + s_total[x], r1 = s_off[x] + (s_total[x] + row_align - 1) / row_align * row_align;
+    for (int r = r0 + threadIdx.x; r < r1; r += blockDim.x) {
+      slot_of_row[r] = -1;
+      if (w_row != nullptr) w_row[r] = 0.f;
     }
   }
+  if (blockIdx.x == gridDim.x - 1) {
+    for (long long r = s_off[E] + threadIdx.x; r < R; r += blockDim.x) {
+      slot_of_row[r] = -1;
+      if (w_row != nullptr) w_row[r] = 0.f;
+    }
+  }
+  for (int e = threadIdx.x; e < E; e += blockDim.x) s_start[e] += s_off[e];
   __syncthreads();
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const long long base = (long long)blockIdx.x * PERM_BLOCK_SLOTS + (long long)w * PERM_ITERS * 32;
-#pragma unroll
-  for (int it = 0; it < PERM_ITERS; ++it) {
-    const long long s = base + it * 32 + lane;
-    const int e = e_reg[it];
-    const uint32_t peers = __match_any_sync(0xffffffffu, e);
-    const int start = (e >= 0) ? warp_cnt[w][e] : 0;
-    __syncwarp();
-    if (e >= 0 && lane == __ffs(peers) - 1) warp_cnt[w][e] = start + __popc(peers);
-    __syncwarp();
-    if (e >= 0) {
-      const int row = start + __popc(peers & lanemask_lt());
-      row_of_slot[s] = row;
-      slot_of_row[row] = (int32_t)s;
-    }
-  }
+  rank_and_write(e_mine, NK, E, slots_per_block, grp_cnt, s_start, row_of_slot, slot_of_row, w, w_row);
 }
 
 // Row gather, one warp per token: the token's row is read once and written to its K rows.  Blocks past the
@@ -470,7 +491,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) gate_wgrad_kernel(const T* __restrict__ Xp, const int32_t* __restrict__ counts,
                                                          const int32_t* __restrict__ offsets,
                                                          const int32_t* __restrict__ slot_of_row,
-                                                         const float* __restrict__ dl, float* __restrict__ dWg, int d) {
+                                                         const float* __restrict__ dl, float* __restrict__ dWg, int d,
+                                                         int accumulate) {
   using V = Vec16<T>;
   __shared__ float part[8][32 * V::N];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -499,7 +521,7 @@ __global__ void __launch_bounds__(256) gate_wgrad_kernel(const T* __restrict__ X
 #pragma unroll
     for (int ww = 0; ww < 8; ++ww) s += part[ww][i];
     const int c = blockIdx.x * 32 * V::N + i;
-    if (c < d) dWg[(size_t)e * d + c] = s;
+    if (c < d) dWg[(size_t)e * d + c] = s + (accumulate ? dWg[(size_t)e * d + c] : 0.f);
   }
 }
 
@@ -540,17 +562,17 @@ __global__ void __launch_bounds__(256) shared_gate_wgrad_kernel(const T* __restr
   }
 }
 
-__global__ void sum_splits_kernel(const float* __restrict__ ws, float* __restrict__ out, int d) {
+__global__ void sum_splits_kernel(const float* __restrict__ ws, float* __restrict__ out, int d, int accumulate) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= d) return;
   float s = 0.f;
   for (int i = 0; i < GWS_SPLITS; ++i) s += ws[(size_t)i * d + c];
-  out[c] = s;
+  out[c] = s + (accumulate ? out[c] : 0.f);
 }
 
 inline int perm_blocks(const c2r_config* cfg) {
-  long long NK = (long long)cfg->N * cfg->K;
-  return (int)((NK + PERM_BLOCK_SLOTS - 1) / PERM_BLOCK_SLOTS);
+  const int tb = perm_tokens_per_block(cfg->K);
+  return (cfg->N + tb - 1) / tb;
 }
 
 size_t permute_ws_bytes(const c2r_config* cfg) {
@@ -611,14 +633,15 @@ __global__ void __launch_bounds__(256) gate_dz_kernel(const float* __restrict__ 
   }
 }
 __global__ void __launch_bounds__(256) gate_wgrad_reduce_kernel(const float* __restrict__ partial, int splits, int E, int d,
-                                                                float* __restrict__ dWg, float* __restrict__ dwsg) {
+                                                                float* __restrict__ dWg, float* __restrict__ dwsg,
+                                                                int accumulate) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   const int e = blockIdx.y;  // 0..E: row E is the shared gate
   if (c >= d) return;
   float acc = 0.f;
   for (int sp = 0; sp < splits; ++sp) acc += partial[((size_t)sp * GW_COLS + e) * d + c];
-  if (e < E) dWg[(size_t)e * d + c] = acc;
-  else if (dwsg != nullptr) dwsg[c] = acc;
+  if (e < E) dWg[(size_t)e * d + c] = acc + (accumulate ? dWg[(size_t)e * d + c] : 0.f);
+  else if (dwsg != nullptr) dwsg[c] = acc + (accumulate ? dwsg[c] : 0.f);
 }
 
 size_t gate_bwd_ws_bytes(const c2r_config* cfg) {
@@ -627,28 +650,34 @@ size_t gate_bwd_ws_bytes(const c2r_config* cfg) {
   return simt > tc ? simt : tc;
 }
 
+// have_hist: block_counts already holds the per-block expert counts of idx in this blocking (the routing
+// kernel wrote them), so the histogram launch is skipped.  w / w_row (both or neither): see rank_and_write.
 template <typename T>
 int permute_impl(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const T* X, int32_t* counts,
                  int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, T* Xp, int32_t* status, void* ws,
-                 cudaStream_t s) {
+                 cudaStream_t s, bool have_hist, const float* w, float* w_row) {
   const long long NK = (long long)cfg->N * cfg->K;
   const long long R = permuted_rows(cfg);
   const int nb = perm_blocks(cfg);
+  const int spb = perm_tokens_per_block(cfg->K) * cfg->K;
   int32_t* block_counts = (int32_t*)ws;
-  C2R_CUDA(cudaMemsetAsync(slot_of_row, 0xFF, sizeof(int32_t) * R, s));
-  if (nb > 0) {
-    perm_hist_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, status, 0);
+  if (w == nullptr) w_row = nullptr;
+  if (nb > 0 && !have_hist) {
+    perm_hist_kernel<<<nb, PERM_THREADS, 0, s>>>(idx, NK, cfg->E, spb, block_counts, status, 0);
     C2R_LAUNCH_CHECK();
   }
   if (nb > 0 && nb <= PERM_FUSED_MAX_BLOCKS) {
-    perm_rank_fused_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, nb, expert_rank, cfg->row_align,
-                                                          counts, offsets, row_of_slot, slot_of_row);
+    perm_rank_fused_kernel<<<nb, PERM_THREADS, 0, s>>>(idx, NK, cfg->E, spb, block_counts, nb, expert_rank, cfg->row_align,
+                                                       R, counts, offsets, row_of_slot, slot_of_row, w, w_row, status);
     C2R_LAUNCH_CHECK();
   } else {
-    perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, cfg->E, expert_rank, cfg->row_align, counts, offsets);
+    C2R_CUDA(cudaMemsetAsync(slot_of_row, 0xFF, sizeof(int32_t) * R, s));
+    if (w_row != nullptr) C2R_CUDA(cudaMemsetAsync(w_row, 0, sizeof(float) * R, s));
+    perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, cfg->E, expert_rank, cfg->row_align, counts, offsets, status);
     C2R_LAUNCH_CHECK();
     if (nb > 0) {
-      perm_rank_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(idx, NK, cfg->E, block_counts, offsets, row_of_slot, slot_of_row, 0);
+      perm_rank_kernel<<<nb, PERM_THREADS, 0, s>>>(idx, NK, cfg->E, spb, block_counts, offsets, row_of_slot, slot_of_row, 0,
+                                                   w, w_row);
       C2R_LAUNCH_CHECK();
     }
   }
@@ -662,7 +691,6 @@ int permute_impl(const c2r_config* cfg, const int32_t* idx, const int32_t* exper
       C2R_LAUNCH_CHECK();
     }
   }
-  (void)R;
   return C2R_OK;
 }
 
@@ -670,19 +698,49 @@ int permute_impl(const c2r_config* cfg, const int32_t* idx, const int32_t* exper
 
 using namespace c2r;
 
-extern "C" int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
-                           int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp,
-                           int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+int c2r::permute_call(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X, int32_t* counts,
+                      int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row, void* Xp, int32_t* status, void* ws,
+                      size_t ws_bytes, void* stream, bool have_hist, const float* w, float* w_row) {
   int rc = check_config(cfg);
   if (rc) return rc;
   C2R_REQUIRE(idx && counts && offsets && row_of_slot && slot_of_row, C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(!X || Xp, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!w_row || w, C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(ws && ws_bytes >= permute_ws_bytes(cfg), C2R_ERR_WORKSPACE);
   if (cfg->dtype == C2R_BF16)
     return permute_impl<__nv_bfloat16>(cfg, idx, expert_rank, (const __nv_bfloat16*)X, counts, offsets, row_of_slot,
-                                       slot_of_row, (__nv_bfloat16*)Xp, status, ws, as_stream(stream));
+                                       slot_of_row, (__nv_bfloat16*)Xp, status, ws, as_stream(stream), have_hist, w, w_row);
   return permute_impl<float>(cfg, idx, expert_rank, (const float*)X, counts, offsets, row_of_slot, slot_of_row,
-                             (float*)Xp, status, ws, as_stream(stream));
+                             (float*)Xp, status, ws, as_stream(stream), have_hist, w, w_row);
+}
+
+extern "C" int c2r_permute(const c2r_config* cfg, const int32_t* idx, const int32_t* expert_rank, const void* X,
+                           const float* w, int32_t* counts, int32_t* offsets, int32_t* row_of_slot, int32_t* slot_of_row,
+                           void* Xp, float* w_row, int32_t* status, void* ws, size_t ws_bytes, int ws_has_histogram,
+                           void* stream) {
+  return permute_call(cfg, idx, expert_rank, X, counts, offsets, row_of_slot, slot_of_row, Xp, status, ws, ws_bytes, stream,
+                      ws_has_histogram != 0 && cfg && cfg->N > 0, w, w_row);
+}
+
+extern "C" int c2r_permute_rows(const c2r_config* cfg, const void* X, const int32_t* row_of_slot, const int32_t* counts,
+                                const int32_t* offsets, void* Xp, void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(X && row_of_slot && counts && offsets && Xp, C2R_ERR_INVALID_ARG);
+  const int token_blocks = (cfg->N + 7) / 8;
+  const int pad_blocks = cfg->row_align > 1 ? cfg->E : 0;
+  if (token_blocks + pad_blocks == 0) return C2R_OK;
+  cudaStream_t s = as_stream(stream);
+  if (cfg->dtype == C2R_BF16)
+    permute_rows_kernel<__nv_bfloat16><<<token_blocks + pad_blocks, 256, 0, s>>>(
+        (const __nv_bfloat16*)X, row_of_slot, (__nv_bfloat16*)Xp, cfg->N, cfg->d, cfg->K, counts, offsets, token_blocks,
+        cfg->row_align);
+  else
+    permute_rows_kernel<float><<<token_blocks + pad_blocks, 256, 0, s>>>((const float*)X, row_of_slot, (float*)Xp, cfg->N,
+                                                                         cfg->d, cfg->K, counts, offsets, token_blocks,
+                                                                         cfg->row_align);
+  C2R_LAUNCH_CHECK();
+  return C2R_OK;
 }
 
 template <typename T>
@@ -701,8 +759,7 @@ extern "C" int c2r_combine(const c2r_config* cfg, const void* Yp, const float* w
                            const void* Ys, const float* z, void* Y, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
-  C2R_REQUIRE(Yp && w && row_of_slot && Y, C2R_ERR_INVALID_ARG);
-  C2R_REQUIRE(!Ys || z, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(Yp && row_of_slot && Y, C2R_ERR_INVALID_ARG);
   if (cfg->dtype == C2R_BF16)
     return gather_sum_launch<__nv_bfloat16>(cfg, Yp, row_of_slot, w, Ys, z, nullptr, nullptr, nullptr, nullptr,
                                             nullptr, Y, 0, as_stream(stream));
@@ -761,7 +818,7 @@ extern "C" int c2r_combine_bwd(const c2r_config* cfg, const void* dY, const void
 template <typename T>
 static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
                            const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
-                           float* dWg, float* dwsg, void* ws, cudaStream_t s) {
+                           float* dWg, float* dwsg, int accumulate, void* ws, cudaStream_t s) {
   using V = Vec16<T>;
   if (sizeof(T) == 2 && X != nullptr && ws != nullptr && cfg->N > 0 && cfg->d % 16 == 0 && cfg->E < GW_COLS &&
       ((uintptr_t)X & 15u) == 0 && tc_supported(cfg, 1, 16, cfg->N)) {
@@ -778,19 +835,19 @@ static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp,
     int rc = tc_gate_wgrad(cfg, X, dLd, partial, g.splits, sc, so, nullptr, s);
     if (rc) return rc;
     gate_wgrad_reduce_kernel<<<dim3((cfg->d + 255) / 256, cfg->E + 1), 256, 0, s>>>(partial, g.splits, cfg->E, cfg->d,
-                                                                                   dWg, dz ? dwsg : nullptr);
+                                                                                   dWg, dz ? dwsg : nullptr, accumulate);
     C2R_LAUNCH_CHECK();
     return C2R_OK;
   }
   C2R_REQUIRE(Xp != nullptr, C2R_ERR_INVALID_ARG);  // the row-serial form walks the permuted rows
   const int colblocks = (cfg->d + 32 * V::N - 1) / (32 * V::N);
   gate_wgrad_kernel<T><<<dim3(colblocks, cfg->E), 256, 0, s>>>((const T*)Xp, counts, offsets, slot_of_row, dl, dWg,
-                                                               cfg->d);
+                                                               cfg->d, accumulate);
   C2R_LAUNCH_CHECK();
   if (dz) {
     shared_gate_wgrad_kernel<T><<<dim3(colblocks, GWS_SPLITS), 256, 0, s>>>((const T*)X, dz, (float*)ws, cfg->N, cfg->d);
     C2R_LAUNCH_CHECK();
-    sum_splits_kernel<<<(cfg->d + 255) / 256, 256, 0, s>>>((const float*)ws, dwsg, cfg->d);
+    sum_splits_kernel<<<(cfg->d + 255) / 256, 256, 0, s>>>((const float*)ws, dwsg, cfg->d, accumulate);
     C2R_LAUNCH_CHECK();
   }
   return C2R_OK;
@@ -798,7 +855,7 @@ static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp,
 
 extern "C" int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
                             const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
-                            float* dWg, float* dwsg, void* ws, size_t ws_bytes, void* stream) {
+                            float* dWg, float* dwsg, int accumulate, void* ws, size_t ws_bytes, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   C2R_REQUIRE(counts && offsets && slot_of_row && dl && dWg, C2R_ERR_INVALID_ARG);
@@ -806,9 +863,10 @@ extern "C" int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp
   C2R_REQUIRE(!dz || (ws && ws_bytes >= gate_bwd_ws_bytes(cfg)), C2R_ERR_WORKSPACE);
   if (ws && ws_bytes < gate_bwd_ws_bytes(cfg)) ws = nullptr;  // too small for the tensor-core form: row-serial kernel
   if (cfg->dtype == C2R_BF16)
-    return gate_bwd_launch<__nv_bfloat16>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws,
+    return gate_bwd_launch<__nv_bfloat16>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, accumulate, ws,
                                           as_stream(stream));
-  return gate_bwd_launch<float>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws, as_stream(stream));
+  return gate_bwd_launch<float>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, accumulate, ws,
+                                as_stream(stream));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -852,16 +910,17 @@ extern "C" int c2r_permute_static(const c2r_config* cfg, const int32_t* idx, con
   if (rc) return rc;
   C2R_REQUIRE(idx && counts && offsets && row_of_slot && slot_of_row, C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(!X || Xp, C2R_ERR_INVALID_ARG);
-  // the scratch holds one int32 per (block of 512 slots, expert)
+  // the scratch holds one int32 per (block of the sort, expert)
   if (permute_ws_bytes(cfg) > C2R_PERMUTE_STATIC_SCRATCH_BYTES) return C2R_ERR_STATIC_SCRATCH;
   int32_t* scratch = nullptr;
   rc = perm_static_scratch(&scratch);
   if (rc) return rc;
   if (cfg->dtype == C2R_BF16)
     return permute_impl<__nv_bfloat16>(cfg, idx, expert_rank, (const __nv_bfloat16*)X, counts, offsets, row_of_slot,
-                                       slot_of_row, (__nv_bfloat16*)Xp, status, scratch, as_stream(stream));
+                                       slot_of_row, (__nv_bfloat16*)Xp, status, scratch, as_stream(stream), false, nullptr,
+                                       nullptr);
   return permute_impl<float>(cfg, idx, expert_rank, (const float*)X, counts, offsets, row_of_slot, slot_of_row,
-                             (float*)Xp, status, scratch, as_stream(stream));
+                             (float*)Xp, status, scratch, as_stream(stream), false, nullptr, nullptr);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -978,24 +1037,26 @@ static int dispatch_dedup_impl(const c2r_config* cfg, const int32_t* idx, const 
   const long long R = permuted_rows(cfg);
   const long long cap = (long long)N * (K < P ? K : P);  // rows the receive side can need
   // the per-expert layout itself (counts, offsets, both row maps) is the plain dispatch's
-  int rc = permute_impl<T>(cfg, idx, expert_rank, nullptr, counts, offsets, row_of_slot, slot_of_row, nullptr, status, ws, s);
+  int rc = permute_impl<T>(cfg, idx, expert_rank, nullptr, counts, offsets, row_of_slot, slot_of_row, nullptr, status, ws, s,
+                           false, nullptr, nullptr);
   if (rc) return rc;
   int32_t* block_counts = (int32_t*)ws;  // free again: the calls above are ordered on the stream
   int32_t* key = (int32_t*)((char*)ws + align256_(permute_ws_bytes(cfg)));
   int32_t* slot_of_recv_row = (int32_t*)((char*)key + align256_(sizeof(int32_t) * (NK > 0 ? NK : 1)));
   const int nb = perm_blocks(cfg);
+  const int spb = perm_tokens_per_block(K) * K;
   if (N > 0) {
     dedup_keys_kernel<<<(N + 255) / 256, 256, 0, s>>>(idx, part, key, N, E, K, P);
     C2R_LAUNCH_CHECK();
     C2R_CUDA(cudaMemsetAsync(slot_of_recv_row, 0xFF, sizeof(int32_t) * NK, s));
-    perm_hist_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(key, NK, P, block_counts, status, 1);
+    perm_hist_kernel<<<nb, PERM_THREADS, 0, s>>>(key, NK, P, spb, block_counts, status, 1);
     C2R_LAUNCH_CHECK();
   }
-  perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, P, nullptr, 1, recv_counts, recv_offsets);
+  perm_scan_kernel<<<1, 1024, 0, s>>>(block_counts, nb, P, nullptr, 1, recv_counts, recv_offsets, nullptr);
   C2R_LAUNCH_CHECK();
   if (N > 0) {
-    perm_rank_kernel<<<nb, PERM_WARPS * 32, 0, s>>>(key, NK, P, block_counts, recv_offsets, recv_row_of_slot,
-                                                    slot_of_recv_row, 1);
+    perm_rank_kernel<<<nb, PERM_THREADS, 0, s>>>(key, NK, P, spb, block_counts, recv_offsets, recv_row_of_slot,
+                                                 slot_of_recv_row, 1, nullptr, nullptr);
     C2R_LAUNCH_CHECK();
     dedup_fill_kernel<<<(N + 255) / 256, 256, 0, s>>>(idx, part, key, recv_row_of_slot, N, E, K, P);
     C2R_LAUNCH_CHECK();

@@ -79,72 +79,105 @@ __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) {
   return (va > vb) || (va == vb && ia < ib);
 }
 
-__global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ L, const uint64_t* __restrict__ mask,
-                                                    int32_t* __restrict__ idx, float* __restrict__ w,
-                                                    float* __restrict__ p, int32_t* __restrict__ status, int N, int E,
-                                                    int K, int renorm) {
-  const int lane = threadIdx.x & 31;
-  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (t >= N) return;
+constexpr int ROUTE_WARPS = 16;
+
+// A block owns tokens_per_block consecutive tokens (the blocking of the dispatch's counting sort), a warp
+// every ROUTE_WARPS-th of them.  block_counts (optional): [blocks][E] experts' slot counts of the block's
+// tokens -- the histogram the dispatch starts from, so it need not read idx again to build it.  A token's
+// K experts are distinct, hence lanes 0..K-1 bump different counters of the warp's private row: no atomics.
+__global__ void __launch_bounds__(ROUTE_WARPS * 32) route_kernel(const float* __restrict__ L, const uint64_t* __restrict__ mask,
+                                                                 int32_t* __restrict__ idx, float* __restrict__ w,
+                                                                 float* __restrict__ p, int32_t* __restrict__ status, int N,
+                                                                 int E, int K, int renorm, int tokens_per_block,
+                                                                 int32_t* __restrict__ block_counts) {
+  __shared__ int warp_cnt[ROUTE_WARPS][64];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (block_counts != nullptr) {
+    for (int i = threadIdx.x; i < ROUTE_WARPS * 64; i += blockDim.x) (&warp_cnt[0][0])[i] = 0;
+    __syncthreads();
+  }
   const float NEG_INF = -INFINITY;
-  float v0 = NEG_INF, v1 = NEG_INF;
+  const int t_end = min(N, (int)(blockIdx.x + 1) * tokens_per_block);
   int flags = 0;
-  if (lane < E) v0 = L[(size_t)t * E + lane];
-  if (lane + 32 < E) v1 = L[(size_t)t * E + lane + 32];
-  if (v0 != v0) { v0 = NEG_INF; flags |= C2R_STATUS_NAN_LOGIT; }
-  if (v1 != v1) { v1 = NEG_INF; flags |= C2R_STATUS_NAN_LOGIT; }
-  uint64_t avail = (E == 64) ? ~0ull : ((1ull << E) - 1ull);
-  const uint64_t valid = avail;
-  uint64_t chosen = 0;
-  float my_sel = NEG_INF;  // lane k keeps the logit picked in round k
-  int my_idx = 0;
-  for (int k = 0; k < K; ++k) {
-    const bool ok0 = (avail >> lane) & 1ull;
-    const bool ok1 = (avail >> (lane + 32)) & 1ull;
-    float bv;
-    int bi;
-    if (ok0 && (!ok1 || v0 >= v1)) { bv = v0; bi = lane; }
-    else if (ok1) { bv = v1; bi = lane + 32; }
-    else { bv = NEG_INF; bi = 1 << 20; }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-      int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-      if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-    }
-    if (bi >= E) {  // candidate set exhausted: fall back to the lowest unselected expert
-      flags |= C2R_STATUS_SET_TOO_SMALL;
-      bi = __ffsll((long long)(valid & ~chosen)) - 1;
-      bv = NEG_INF;
-    }
-    chosen |= 1ull << bi;
-    avail &= ~(1ull << bi);
-    if (k == 0 && mask != nullptr) avail &= mask[bi];
-    if (lane == k) { my_sel = bv; my_idx = bi; }
+  int t = blockIdx.x * tokens_per_block + warp;
+  float n0 = NEG_INF, n1 = NEG_INF;  // the next token's logits, requested one token ahead
+  if (t < t_end) {
+    if (lane < E) n0 = L[(size_t)t * E + lane];
+    if (lane + 32 < E) n1 = L[(size_t)t * E + lane + 32];
   }
-  // Eq. 1 weights.  The round-0 logit is the row maximum, so it is the softmax shift for both forms.
-  const float top = __shfl_sync(0xffffffffu, my_sel, 0);
-  float denom;
-  if (renorm) {
-    float ek = (lane < K) ? expf(my_sel - top) : 0.f;
-    denom = ek;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, off);
-    if (lane < K) w[(size_t)t * K + lane] = ek / denom;
-  }
-  if (!renorm || p != nullptr) {
-    float e0 = (lane < E) ? expf(v0 - top) : 0.f;
-    float e1 = (lane + 32 < E) ? expf(v1 - top) : 0.f;
-    float s = e0 + e1;
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-    if (p != nullptr) {
-      if (lane < E) p[(size_t)t * E + lane] = e0 / s;
-      if (lane + 32 < E) p[(size_t)t * E + lane + 32] = e1 / s;
+  for (; t < t_end; t += ROUTE_WARPS) {
+    float v0 = n0, v1 = n1;
+    if (t + ROUTE_WARPS < t_end) {
+      if (lane < E) n0 = L[(size_t)(t + ROUTE_WARPS) * E + lane];
+      if (lane + 32 < E) n1 = L[(size_t)(t + ROUTE_WARPS) * E + lane + 32];
     }
-    if (!renorm && lane < K) w[(size_t)t * K + lane] = expf(my_sel - top) / s;
+    if (v0 != v0) { v0 = NEG_INF; flags |= C2R_STATUS_NAN_LOGIT; }
+    if (v1 != v1) { v1 = NEG_INF; flags |= C2R_STATUS_NAN_LOGIT; }
+    uint64_t avail = (E == 64) ? ~0ull : ((1ull << E) - 1ull);
+    const uint64_t valid = avail;
+    uint64_t chosen = 0;
+    float my_sel = NEG_INF;  // lane k keeps the logit picked in round k
+    int my_idx = 0;
+    for (int k = 0; k < K; ++k) {
+      const bool ok0 = (avail >> lane) & 1ull;
+      const bool ok1 = (avail >> (lane + 32)) & 1ull;
+      float bv;
+      int bi;
+      if (ok0 && (!ok1 || v0 >= v1)) { bv = v0; bi = lane; }
+      else if (ok1) { bv = v1; bi = lane + 32; }
+      else { bv = NEG_INF; bi = 1 << 20; }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+        int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+        if (better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+      }
+      if (bi >= E) {  // candidate set exhausted: fall back to the lowest unselected expert
+        flags |= C2R_STATUS_SET_TOO_SMALL;
+        bi = __ffsll((long long)(valid & ~chosen)) - 1;
+        bv = NEG_INF;
+      }
+      chosen |= 1ull << bi;
+      avail &= ~(1ull << bi);
+      if (k == 0 && mask != nullptr) avail &= mask[bi];
+      if (lane == k) { my_sel = bv; my_idx = bi; }
+    }
+    // Eq. 1 weights.  The round-0 logit is the row maximum, so it is the softmax shift for both forms.
+    const float top = __shfl_sync(0xffffffffu, my_sel, 0);
+    float denom;
+    if (renorm) {
+      float ek = (lane < K) ? expf(my_sel - top) : 0.f;
+      denom = ek;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) denom += __shfl_xor_sync(0xffffffffu, denom, off);
+      if (lane < K) w[(size_t)t * K + lane] = ek / denom;
+    }
+    if (!renorm || p != nullptr) {
+      float e0 = (lane < E) ? expf(v0 - top) : 0.f;
+      float e1 = (lane + 32 < E) ? expf(v1 - top) : 0.f;
+      float s = e0 + e1;
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+      if (p != nullptr) {
+        if (lane < E) p[(size_t)t * E + lane] = e0 / s;
+        if (lane + 32 < E) p[(size_t)t * E + lane + 32] = e1 / s;
+      }
+      if (!renorm && lane < K) w[(size_t)t * K + lane] = expf(my_sel - top) / s;
+    }
+    if (lane < K) {
+      idx[(size_t)t * K + lane] = my_idx;
+      if (block_counts != nullptr) warp_cnt[warp][my_idx] += 1;
+    }
   }
-  if (lane < K) idx[(size_t)t * K + lane] = my_idx;
+  if (block_counts != nullptr) {
+    __syncthreads();
+    for (int e = threadIdx.x; e < E; e += blockDim.x) {
+      int s = 0;
+#pragma unroll
+      for (int x = 0; x < ROUTE_WARPS; ++x) s += warp_cnt[x][e];
+      block_counts[(size_t)blockIdx.x * E + e] = s;
+    }
+  }
   if (status != nullptr) {
     flags = __reduce_or_sync(0xffffffffu, flags);
     if (flags && lane == 0) atomicOr(status, flags);
@@ -158,6 +191,42 @@ __global__ void route_bwd_kernel(const float* __restrict__ w, const float* __res
   float s = 0.f;
   for (int k = 0; k < K; ++k) s = fmaf(w[(size_t)t * K + k], dw[(size_t)t * K + k], s);
   for (int k = 0; k < K; ++k) dl[(size_t)t * K + k] = w[(size_t)t * K + k] * (dw[(size_t)t * K + k] - s);
+}
+
+// Backward of the Eq. 1 weights when the experts applied them themselves (row-scaled SwiGLU): the backward
+// GEMM left, per permuted row, partial dots whose sum is q = s_r <dH_r, H_r / s_r> = w dL/dw.  With
+// S = sum_j q_j:  dl_k = w_k (dw_k - sum_j w_j dw_j) = q_k - w_k S  -- no division by a weight that may be 0.
+// dw (optional, informational) = q_k / w_k where w_k > 0.  Shared expert: q_s = g dL/dg, dz = q_s (1 - g).
+// Partials are added in index order.
+__global__ void __launch_bounds__(256) route_bwd_scaled_kernel(const float* __restrict__ w,
+                                                               const int32_t* __restrict__ row_of_slot,
+                                                               const float* __restrict__ qpart, int nq, long long R,
+                                                               const float* __restrict__ z,
+                                                               const float* __restrict__ qspart, int nqs,
+                                                               float* __restrict__ dw, float* __restrict__ dl,
+                                                               float* __restrict__ dz, int N, int K) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= N) return;
+  float q[8];
+  float S = 0.f;
+  for (int k = 0; k < K; ++k) {
+    const long long row = row_of_slot[(size_t)t * K + k];
+    float acc = 0.f;
+    for (int j = 0; j < nq; ++j) acc += qpart[(long long)j * R + row];
+    q[k] = acc;
+    S += acc;
+  }
+  for (int k = 0; k < K; ++k) {
+    const float wk = w[(size_t)t * K + k];
+    dl[(size_t)t * K + k] = q[k] - wk * S;
+    if (dw != nullptr) dw[(size_t)t * K + k] = wk > 0.f ? q[k] / wk : 0.f;
+  }
+  if (dz != nullptr) {
+    float acc = 0.f;
+    for (int j = 0; j < nqs; ++j) acc += qspart[(long long)j * N + t];
+    const float g = 1.0f / (1.0f + expf(-z[t]));
+    dz[t] = acc * (1.0f - g);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -322,16 +391,36 @@ extern "C" int c2r_gate_logits(const c2r_config* cfg, const void* X, const void*
   return gate_logits_impl(cfg, X, Wg, wsg, L, z, nullptr, stream);
 }
 
-extern "C" int c2r_route(const c2r_config* cfg, const float* L, const uint64_t* mask, int32_t* idx, float* w, float* p,
-                         int32_t* status, void* stream) {
+int c2r::route_impl(const c2r_config* cfg, const float* L, const uint64_t* mask, int32_t* idx, float* w, float* p,
+                    int32_t* status, int32_t* block_counts, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   C2R_REQUIRE(L && idx && w, C2R_ERR_INVALID_ARG);
   if (mask) C2R_REQUIRE(cfg->T >= cfg->K - 1 && cfg->T <= cfg->E - 1, C2R_ERR_INVALID_ARG);
   if (cfg->N == 0) return C2R_OK;
-  const int warps = 8;
-  route_kernel<<<(cfg->N + warps - 1) / warps, warps * 32, 0, as_stream(stream)>>>(L, mask, idx, w, p, status, cfg->N,
-                                                                                 cfg->E, cfg->K, cfg->renorm);
+  const int tpb = perm_tokens_per_block(cfg->K);
+  route_kernel<<<(cfg->N + tpb - 1) / tpb, ROUTE_WARPS * 32, 0, as_stream(stream)>>>(L, mask, idx, w, p, status, cfg->N, cfg->E,
+                                                                                   cfg->K, cfg->renorm, tpb, block_counts);
+  C2R_LAUNCH_CHECK();
+  return C2R_OK;
+}
+
+extern "C" int c2r_route(const c2r_config* cfg, const float* L, const uint64_t* mask, int32_t* idx, float* w, float* p,
+                         int32_t* status, void* permute_ws, void* stream) {
+  return route_impl(cfg, L, mask, idx, w, p, status, (int32_t*)permute_ws, stream);
+}
+
+extern "C" int c2r_route_bwd_scaled(const c2r_config* cfg, const float* w, const int32_t* row_of_slot, const float* qpart,
+                                    int nq, const float* z, const float* qspart, int nqs, float* dw, float* dl, float* dz,
+                                    void* stream) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  C2R_REQUIRE(w && row_of_slot && qpart && dl && nq >= 0, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(!dz || (z && qspart && nqs >= 0), C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(cfg->renorm == 1, C2R_ERR_UNSUPPORTED_SHAPE);
+  if (cfg->N == 0) return C2R_OK;
+  route_bwd_scaled_kernel<<<(cfg->N + 255) / 256, 256, 0, as_stream(stream)>>>(w, row_of_slot, qpart, nq, permuted_rows(cfg),
+                                                                              z, qspart, nqs, dw, dl, dz, cfg->N, cfg->K);
   C2R_LAUNCH_CHECK();
   return C2R_OK;
 }

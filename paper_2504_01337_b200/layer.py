@@ -21,7 +21,7 @@ class C2RLayer:
     to torch tensors."""
 
     def __init__(self, N, d, E, I, K, T, P, I_s=0, bf16=True, row_align=None, backward=True, profile=False,
-                 renorm=1, device="cuda", gather_fused=False):
+                 renorm=1, device="cuda", gather_fused=False, side_stream=False):
         if row_align is None:
             row_align = 128 if bf16 else 1
         self.cfg = B.make_config(N, d, E, I, K, T, P, I_s, B.BF16 if bf16 else B.F32, row_align, renorm,
@@ -45,6 +45,7 @@ class C2RLayer:
         t["offsets"] = buf((E + 1,), i32)
         t["row_of_slot"] = buf((N * K,), i32)
         t["slot_of_row"] = buf((R,), i32)
+        t["w_row"] = buf((R,), f32)
         if not (gather_fused and bf16):  # the gather-fused GEMMs read token rows from X: no permuted copy
             t["Xp"] = buf((R, d))
         t["H"] = buf((R, I))
@@ -74,13 +75,19 @@ class C2RLayer:
             t["dWg"] = buf((E, d), f32)
             t["dX"] = buf((N, d))
             if I_s:
-                t["dYs"] = buf((N, d))
                 t["dABs"] = buf((N, 2 * I_s))
                 t["dXs"] = buf((N, d), f32)
                 t["dz"] = buf((N,), f32)
                 t["dWs13p"] = buf((1, 2 * I_s, d))
                 t["dWs2"] = buf((1, d, I_s))
                 t["dwsg"] = buf((d,), f32)
+        if side_stream and I_s:
+            # the shared expert's GEMMs go to a second stream between a fork from and a join into the caller's
+            with torch.cuda.device(dev):
+                t["stream2"] = torch.cuda.Stream()
+                t["ev_fork"], t["ev_join"] = torch.cuda.Event(), torch.cuda.Event()
+                # an event has no handle before its first record
+                t["ev_fork"].record(); t["ev_join"].record()
         if profile:
             t["C"] = torch.zeros((E, E), dtype=i32, device=dev)
             t["I_T"] = torch.zeros((E, max(T, 1)), dtype=i32, device=dev)

@@ -104,21 +104,24 @@ def _check_sampled_tokens(wl, lay, X, dY, L, idx, sets, rank, n_sample):
     assert np.array_equal(f["idx"], idx[S])
     rows_dev = lay.host("row_of_slot").reshape(wl.N, K)[S].reshape(-1)
     rows_ref = f["row_of_slot"].reshape(-1)
-    assert_close_elem(_dev_rows(lay.t["H"], rows_dev), f["H"][rows_ref], what="H")
-    assert_close_rms(_dev_rows(lay.t["Yp"], rows_dev), f["Yp"][rows_ref], 5e-2, "Yp", out_bf16=False)
+    # the library applies the Eq. 1 weight of a slot inside the expert call: its H and Yp carry it
+    ws = f["w"].reshape(-1)[:, None]
+    assert_close_abs(_dev_rows(lay.t["w_row"], rows_dev), ws[:, 0], 1e-5, "w_row")
+    assert_close_elem(_dev_rows(lay.t["H"], rows_dev), ws * f["H"][rows_ref], what="H")
+    assert_close_rms(_dev_rows(lay.t["Yp"], rows_dev), ws * f["Yp"][rows_ref], 5e-2, "Yp", out_bf16=False)
     assert np.array_equal(_dev_rows(lay.t["Xp"], rows_dev), X[S].astype(np.float64).repeat(K, axis=0))
     assert_close_rms(_dev_rows(lay.t["Y"], S), f["Y"], 2e-2, "Y")
     g = O.layer_bwd(X[S], Wg, W1, W3, W2, f, dY[S], shared=sh, wsg=wsg)
     assert_close_rms(_dev_rows(lay.t["dw"], S), g["dw"], 2e-2, "dw", out_bf16=False)
     dl_ref = np.take_along_axis(g["dL"], f["idx"], axis=1)
     assert_close_rms(_dev_rows(lay.t["dl"], S), dl_ref, 2e-2, "dl", out_bf16=False)
-    assert_close_elem(_dev_rows(lay.t["dYp"], rows_dev), g["dYp"][rows_ref], what="dYp")
+    assert np.array_equal(_dev_rows(lay.t["dYp"], rows_dev), dY[S].astype(np.float64).repeat(K, axis=0))
     assert_close_rms(_dev_rows(lay.t["dXp"], rows_dev), g["dXp"][rows_ref], 5e-2, "dXp", out_bf16=False)
     assert_close_rms(_dev_rows(lay.t["dX"], S), g["dX"], 2e-2, "dX")
     if wl.I_s:
         assert_close_abs(_dev_rows(lay.t["z"], S), f["z"], 1e-4, "z")
         assert_close_rms(_dev_rows(lay.t["dz"], S), g["dz"], 2e-2, "dz", out_bf16=False)
-        assert_close_rms(_dev_rows(lay.t["Ys"], S), f["Ys"], 5e-2, "Ys", out_bf16=False)
+        assert_close_rms(_dev_rows(lay.t["Ys"], S), O.sigmoid(f["z"])[:, None] * f["Ys"], 5e-2, "Ys", out_bf16=False)
 
 
 def _check_expert_grads(wl, lay, X, dY, w_ref, counts, offsets, sor, experts):
@@ -135,7 +138,7 @@ def _check_expert_grads(wl, lay, X, dY, w_ref, counts, offsets, sor, experts):
         cnt, off = np.array([n]), np.array([0, n])
         A, B, H, _ = O.swiglu_fwd(Xe, cnt, off, W1[e:e + 1], W3[e:e + 1], W2[e:e + 1])
         dXp, dW1, dW3, dW2 = O.swiglu_bwd(Xe, cnt, off, W1[e:e + 1], W3[e:e + 1], W2[e:e + 1], A, B, dYpe)
-        assert_close_elem(lay.t["H"][r0:r0 + n].float().cpu().numpy(), H, what=f"H[{e}]")
+        assert_close_elem(lay.t["H"][r0:r0 + n].float().cpu().numpy(), w_ref[tok, k][:, None] * H, what=f"H[{e}]")
         assert_close_rms(lay.t["dXp"][r0:r0 + n].cpu().numpy(), dXp, 5e-2, f"dXp[{e}]", out_bf16=False)
         # error scale of each gradient element: sqrt(sum over the expert's rows of (term)^2), see assert_close_contraction
         sg = O.sigmoid(A)
@@ -162,7 +165,7 @@ def _check_shared_slabs(wl, lay, X, dY, slabs, width=64):
         sl = slice(j0, j0 + width)
         A, B, H, _ = O.dense_swiglu(X64, Ws1[sl], Ws3[sl], Ws2[:, sl])
         _, dW1, dW3, dW2 = O.dense_swiglu_bwd(X64, Ws1[sl], Ws3[sl], Ws2[:, sl], A, B, dYs)
-        assert_close_elem(lay.t["Hs"][:, sl].float().cpu().numpy(), H, what=f"Hs[:, {j0}:]")
+        assert_close_elem(lay.t["Hs"][:, sl].float().cpu().numpy(), O.sigmoid(z)[:, None] * H, what=f"Hs[:, {j0}:]")
         assert_close_rms(d1_dev[sl].float().cpu().numpy(), dW1, 2e-2, f"dWs1[{j0}:]")
         assert_close_rms(d3_dev[sl].float().cpu().numpy(), dW3, 2e-2, f"dWs3[{j0}:]")
         assert_close_rms(lay.t["dWs2"][0][:, sl].float().cpu().numpy(), dW2, 2e-2, f"dWs2[:, {j0}:]")

@@ -5,7 +5,7 @@ import torch
 
 from oracle import c2r_oracle as O
 from paper_2504_01337_b200 import inputs as G
-from tests.util import assert_close_abs, assert_close_elem, assert_close_rms, dev, host, live_rows, mask_of, random_sets
+from tests.util import row_tokens, row_weights, assert_close_abs, assert_close_elem, assert_close_rms, dev, host, live_rows, mask_of, random_sets
 
 pytestmark = pytest.mark.gpu
 
@@ -91,8 +91,10 @@ def test_c1_layer_forward_fp32():
     assert_close_abs(lay.host("w"), f["w"], 1e-4, "w")
     n = f["slot_of_row"].size
     assert np.array_equal(lay.host("Xp")[:n], f["Xp"].astype(np.float32))
-    assert_close_abs(lay.host("H")[:n], f["H"], 1e-4, "H")
-    assert_close_abs(lay.host("Yp")[:n], f["Yp"], 1e-4, "Yp")
+    wr = row_weights(f)[:, None]   # the library applies the Eq. 1 weight of a row inside the expert call
+    assert_close_abs(lay.host("w_row")[:n], wr[:, 0], 1e-6, "w_row")
+    assert_close_abs(lay.host("H")[:n], wr * f["H"], 1e-4, "H")
+    assert_close_abs(lay.host("Yp")[:n], wr * f["Yp"], 1e-4, "Yp")
     assert_close_abs(lay.host("Y"), f["Y"], 1e-4, "Y")
     v = O.dispatch_volume(f["idx"], part_ref, wl.P)
     vol = lay.host("volume")
@@ -139,10 +141,13 @@ def test_small_layer_forward_backward(name, N, d, E, I, K, T, P, I_s, bf16):
     live = live_rows(f["counts"], f["offsets"])
     close32 = _close(bf16, stored_bf16=False)      # results the library keeps in fp32
     mid = (lambda g, r, what: assert_close_elem(g, r, what=what)) if bf16 else close
-    mid(lay.host("H")[live], f["H"][live], "H")
+    wr = row_weights(f)[:, None]   # the library applies the Eq. 1 weight of a row inside the expert call
+    mid(lay.host("H")[live], (wr * f["H"])[live], "H")
     # per-(token, expert) partials are internal: looser max bound, same RMS bound
     part = (lambda g, r, what: assert_close_rms(g, r, 5e-2, what, out_bf16=False)) if bf16 else close
-    part(lay.host("Yp")[live], f["Yp"][live], "Yp")
+    part(lay.host("Yp")[live], (wr * f["Yp"])[live], "Yp")
+    if I_s:
+        part(lay.host("Ys"), O.sigmoid(f["z"])[:, None] * f["Ys"], "Ys")
     close(lay.host("Y"), f["Y"], "Y")
     # backward: the oracle differentiates its own forward (logits from X Wg, routing frozen)
     f2 = O.layer_fwd(X, Wg, W1, W3, W2, sets, K, expert_rank=rank, row_align=align, shared=sh, wsg=wsg)
@@ -150,7 +155,8 @@ def test_small_layer_forward_backward(name, N, d, E, I, K, T, P, I_s, bf16):
         pytest.skip("fp32 and fp64 logits disagree on a near-tie; backward parity needs equal routing")
     g = O.layer_bwd(X, Wg, W1, W3, W2, f2, dY, shared=sh, wsg=wsg)
     close32(lay.host("dw"), g["dw"], "dw")
-    mid(lay.host("dYp")[live], g["dYp"][live], "dYp")
+    # the permuted output gradient is the token's dY, unchanged (the weight enters inside the backward GEMM)
+    assert np.array_equal(lay.host("dYp")[live], dY.astype(np.float32)[row_tokens(f, K)[live]])
     part(lay.host("dXp")[live], g["dXp"][live], "dXp")
     grads = [host(t) for t in lay.unpacked_grads()]
     close(grads[0], g["dW1"], "dW1")
@@ -243,7 +249,7 @@ def test_edge_shapes_bf16_tensor_core_path(name, N, d, E, I, K, T, P, I_s):
     f = O.layer_fwd(X, Wg, W1, W3, W2, sets if T > 0 else None, K, row_align=lay.cfg.row_align, shared=sh, wsg=wsg, logits=Lg)
     assert np.array_equal(lay.host("idx"), f["idx"])
     live = live_rows(f["counts"], f["offsets"])
-    assert_close_elem(lay.host("H")[live], f["H"][live], what="H")
+    assert_close_elem(lay.host("H")[live], (row_weights(f)[:, None] * f["H"])[live], what="H")
     assert_close_rms(lay.host("Y"), f["Y"], 2e-2, "Y")
     f2 = O.layer_fwd(X, Wg, W1, W3, W2, sets if T > 0 else None, K, row_align=lay.cfg.row_align, shared=sh, wsg=wsg)
     if not np.array_equal(f2["idx"], f["idx"]):
@@ -325,3 +331,69 @@ def test_gather_fused_dispatch_is_bit_identical(N, d, E, I, K, T, P, I_s):
         assert torch.equal(plain.t[name], fused.t[name]), name
     for name in ("H", "AB", "Yp", "dAB", "dXp"):  # rows of the layout (beyond its end nothing is written)
         assert torch.equal(plain.t[name][:n_rows], fused.t[name][:n_rows]), name
+    # and the gather-fused run against the oracle itself, on a sample of tokens at the large shape
+    S = np.arange(N) if N <= 2048 else np.sort(np.random.default_rng(1).choice(N, 256, replace=False))
+    Lg = fused.host("L")
+    f = O.layer_fwd(X[S], Wg, W1, W3, W2, sets, K, expert_rank=rank, row_align=1, shared=sh, wsg=wsg, logits=Lg[S])
+    assert np.array_equal(fused.host("idx")[S], f["idx"])
+    assert_close_rms(fused.host("Y")[S], f["Y"], 2e-2, "Y (gather-fused)")
+    f2 = O.layer_fwd(X[S], Wg, W1, W3, W2, sets, K, expert_rank=rank, row_align=1, shared=sh, wsg=wsg)
+    same = np.all(f2["idx"] == f["idx"], axis=1)
+    assert same.mean() > 0.9
+    g = O.layer_bwd(X[S], Wg, W1, W3, W2, f2, dY[S], shared=sh, wsg=wsg)
+    assert_close_rms(fused.host("dX")[S][same], g["dX"][same], 2e-2, "dX (gather-fused)")
+
+
+def test_side_stream_for_the_shared_expert_changes_nothing():
+    """With a second stream the shared expert's GEMMs overlap the routing chain; every result stays bit-identical."""
+    wl = G.Workload("ss", N=3000, d=256, E=8, I=272, K=2, T=4, P=2, I_s=400, bf16=True, seed=17)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    out = []
+    for side in (False, True):
+        lay = _layer(wl, backward=True, profile=True, side_stream=side)
+        lay.set_params(Wg, W1, W3, W2, wsg, G.shared_weights(wl))
+        lay.set_routing(mask=mask_of(random_sets(wl.E, wl.T, seed=3), wl.E))
+        lay.set_input(X, dY)
+        for _ in range(3):
+            lay.train_step()
+        torch.cuda.synchronize()
+        assert int(lay.t["status"].item()) == 0
+        assert ("stream2" in lay.t) == side
+        out.append(lay)
+    a, b = out
+    for name in ("Y", "dX", "dW13p", "dW2", "dWs13p", "dWs2", "dWg", "dwsg", "dz", "dl", "Ys", "dXs", "C", "mask_next"):
+        assert torch.equal(a.t[name], b.t[name]), name
+
+
+def test_two_micro_batches_accumulate_every_parameter_gradient():
+    """accumulate != 0 over a second micro-batch: every parameter gradient (experts, shared expert, gate matrix,
+    shared gate vector) equals the oracle's sum over both micro-batches."""
+    wl = G.Workload("mb", N=512, d=128, E=4, I=144, K=2, T=2, P=2, I_s=64, bf16=False, seed=8)
+    Wg, wsg = G.gate_weights(wl)
+    Wg = Wg * 8
+    W1, W3, W2 = G.expert_weights(wl)
+    sh = G.shared_weights(wl)
+    sets = random_sets(wl.E, wl.T, seed=4)
+    lay = _layer(wl, backward=True)
+    lay.set_params(Wg, W1, W3, W2, wsg, sh)
+    lay.set_routing(mask=mask_of(sets, wl.E))
+    total = None
+    for mb in range(2):
+        wl_mb = G.Workload("mb", N=wl.N, d=wl.d, E=wl.E, I=wl.I, K=wl.K, T=wl.T, P=wl.P, I_s=wl.I_s, bf16=False, seed=8 + 100 * mb)
+        X, dY = G.hidden(wl_mb), G.grad_out(wl_mb)
+        lay.set_input(X, dY)
+        lay.forward()
+        lay.backward(accumulate=mb > 0)
+        torch.cuda.synchronize()
+        f = O.layer_fwd(X, Wg, W1, W3, W2, sets, wl.K, shared=sh, wsg=wsg)
+        assert np.array_equal(lay.host("idx"), f["idx"])
+        g = O.layer_bwd(X, Wg, W1, W3, W2, f, dY, shared=sh, wsg=wsg)
+        keys = ("dW1", "dW3", "dW2", "dWg", "dWs1", "dWs3", "dWs2", "dwsg")
+        total = {k: g[k] if total is None else total[k] + g[k] for k in keys}
+        assert_close_abs(lay.host("dX"), g["dX"], 1e-4, "dX is overwritten, not accumulated")
+    grads = [host(t) for t in lay.unpacked_grads()]
+    for got, k in ((grads[0], "dW1"), (grads[1], "dW3"), (lay.host("dW2"), "dW2"), (lay.host("dWg"), "dWg"),
+                   (grads[2], "dWs1"), (grads[3], "dWs3"), (lay.host("dWs2")[0], "dWs2"), (lay.host("dwsg"), "dwsg")):
+        assert_close_abs(got, total[k], 2e-4, k)

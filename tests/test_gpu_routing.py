@@ -164,6 +164,120 @@ def test_permute_index_and_rows(E, K, N, align):
             assert int(status.item()) == 0
 
 
+def _permute_index_only(b, idx, rank, E, K, N, align, d=64, bf16=True):
+    cfg = b.make_config(N, d, E, 16, K, K - 1, 1, 0, b.BF16 if bf16 else b.F32, align)
+    R = b.permuted_rows(cfg)
+    out = dict(counts=torch.full((E,), -7, dtype=torch.int32, device="cuda"),
+               offsets=torch.full((E + 1,), -7, dtype=torch.int32, device="cuda"),
+               ros=torch.full((N * K,), -7, dtype=torch.int32, device="cuda"),
+               sor=torch.full((R,), -7, dtype=torch.int32, device="cuda"),
+               status=torch.zeros(1, dtype=torch.int32, device="cuda"))
+    ws = torch.empty(b.workspace_bytes(cfg, b.WS_PERMUTE), dtype=torch.uint8, device="cuda")
+    b.permute(cfg, dev(idx.astype(np.int32)), None if rank is None else dev(np.asarray(rank).astype(np.int32)), None,
+              out["counts"], out["offsets"], out["ros"], out["sor"], None, out["status"], ws)
+    return cfg, out
+
+
+def _assert_index_equal(out, ref):
+    rc, ro, rros, rsor = ref
+    assert np.array_equal(host(out["counts"]), rc) and np.array_equal(host(out["offsets"]), ro)
+    assert np.array_equal(host(out["ros"]), rros)
+    got_sor = host(out["sor"])
+    assert np.array_equal(got_sor[: rsor.size], rsor) and np.all(got_sor[rsor.size:] == -1)
+
+
+@pytest.mark.parametrize("E,K,N,align", [(60, 4, 131073, 128), (64, 8, 65600, 128), (7, 3, 164000, 1)])
+def test_permute_large_batch_takes_the_separate_scan(E, K, N, align):
+    """More than 1024 blocks of the sort: histogram, one-block scan and rank run as separate launches."""
+    b = B()
+    assert -(-N // [0, 512, 256, 160, 128, 96, 80, 64, 64][K]) > 1024
+    rng = np.random.default_rng(N)
+    # skewed expert popularity so that the segments differ a lot in length
+    pop = rng.random(E) ** 3 + 1e-3
+    idx = np.stack([rng.choice(E, K, replace=False, p=pop / pop.sum()) for _ in range(2048)])
+    idx = idx[rng.integers(0, 2048, N)]
+    rank = rng.permutation(E)
+    cfg, out = _permute_index_only(b, idx, rank, E, K, N, align)
+    _assert_index_equal(out, O.permute_index(idx, E, rank, align))
+    assert int(out["status"].item()) == 0
+
+
+def test_permute_large_batch_rows():
+    """The separate-scan path with the row gather (small d keeps the buffers small)."""
+    b = B()
+    E, K, N, d, align = 60, 4, 131200, 16, 128
+    rng = np.random.default_rng(5)
+    idx = np.argsort(-rng.standard_normal((N, E)), axis=1, kind="stable")[:, :K]
+    X = G.round_bf16(G.normal(3, G.S_X, (N, d)))
+    cfg = b.make_config(N, d, E, 16, K, K - 1, 1, 0, b.BF16, align)
+    R = b.permuted_rows(cfg)
+    counts = torch.zeros(E, dtype=torch.int32, device="cuda")
+    offsets = torch.zeros(E + 1, dtype=torch.int32, device="cuda")
+    ros = torch.zeros(N * K, dtype=torch.int32, device="cuda")
+    sor = torch.zeros(R, dtype=torch.int32, device="cuda")
+    Xp = torch.full((R, d), 3.0, dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(b.workspace_bytes(cfg, b.WS_PERMUTE), dtype=torch.uint8, device="cuda")
+    b.permute(cfg, dev(idx.astype(np.int32)), None, dev(X, torch.bfloat16), counts, offsets, ros, sor, Xp, None, ws)
+    rc, ro, rros, rsor = O.permute_index(idx, E, None, align)
+    assert np.array_equal(host(ros), rros) and np.array_equal(host(sor)[: rsor.size], rsor)
+    assert np.array_equal(host(Xp)[: rsor.size], O.permute(X, rsor, K))
+
+
+@pytest.mark.parametrize("N", [3000, 140000])
+def test_permute_rejects_a_rank_table_that_is_no_permutation(N):
+    """A duplicated or out-of-range expert_rank entry: identity layout order and the status bit, both in
+    the fused rank kernel (small batch) and in the one-block scan (large batch)."""
+    b = B()
+    E, K = 12, 4
+    rng = np.random.default_rng(N)
+    idx = np.argsort(-rng.standard_normal((N, E)), axis=1, kind="stable")[:, :K]
+    for bad in ([0, 1, 2, 3, 4, 5, 5, 7, 8, 9, 10, 11], [0, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 12],
+                [-1, 1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11]):
+        cfg, out = _permute_index_only(b, idx, bad, E, K, N, 8)
+        assert int(out["status"].item()) & 4
+        _assert_index_equal(out, O.permute_index(idx, E, None, 8))
+    good = rng.permutation(E)
+    cfg, out = _permute_index_only(b, idx, good, E, K, N, 8)
+    assert int(out["status"].item()) == 0
+    _assert_index_equal(out, O.permute_index(idx, E, good, 8))
+
+
+@pytest.mark.parametrize("E,K,N", [(60, 4, 16384), (8, 3, 1000), (64, 8, 70000), (5, 1, 700), (16, 5, 97)])
+def test_route_hands_its_histogram_to_permute(E, K, N):
+    """c2r_route can leave the dispatch's per-block expert histogram in the permute workspace; c2r_permute then
+    skips its own histogram pass.  Same index as the oracle's, and the row weights follow the rows."""
+    b = B()
+    T = min(E - 1, K + 3)
+    L = G.random_logits(N + E, N, E, std=1.5)
+    sets = random_sets(E, T, seed=K)
+    rank = np.random.default_rng(N).permutation(E)
+    cfg = b.make_config(N, 64, E, 16, K, T, 1, 0, b.BF16, 128)
+    R = b.permuted_rows(cfg)
+    idx = torch.zeros((N, K), dtype=torch.int32, device="cuda")
+    w = torch.zeros((N, K), device="cuda")
+    ws = torch.zeros(b.workspace_bytes(cfg, b.WS_PERMUTE), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.route(cfg, dev(L), dev(mask_of(sets, E).view(np.int64)), idx, w, None, status, ws)
+    counts = torch.zeros(E, dtype=torch.int32, device="cuda")
+    offsets = torch.zeros(E + 1, dtype=torch.int32, device="cuda")
+    ros = torch.zeros(N * K, dtype=torch.int32, device="cuda")
+    sor = torch.zeros(R, dtype=torch.int32, device="cuda")
+    w_row = torch.full((R,), 9.0, device="cuda")
+    b.permute(cfg, idx, dev(rank.astype(np.int32)), None, counts, offsets, ros, sor, None, status, ws, w, w_row, True)
+    ridx, rw = O.c2r_route(L, sets, K)
+    assert np.array_equal(host(idx), ridx)
+    ref = O.permute_index(ridx, E, rank, 128)
+    _assert_index_equal(dict(counts=counts, offsets=offsets, ros=ros, sor=sor), ref)
+    want = np.zeros(R, dtype=np.float32)
+    live = ref[3] >= 0
+    want[: ref[3].size][live] = host(w).reshape(-1)[ref[3][live]]
+    if -(-N // [0, 512, 256, 160, 128, 96, 80, 64, 64][K]) <= 1024:
+        assert np.array_equal(host(w_row), want)          # rows without a slot are zeroed by the rank kernel
+    else:
+        assert np.array_equal(host(w_row)[: ref[3].size], want[: ref[3].size])
+    assert int(status.item()) == 0
+
+
 def test_permute_empty_batch_and_bad_index():
     b = B()
     E, K, d = 8, 2, 32

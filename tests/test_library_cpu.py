@@ -47,13 +47,13 @@ def test_sizes_and_argument_checks_need_no_gpu(b):
     cfg = b.make_config(16384, 2048, 60, 1408, 4, 16, 4, 5632, b.BF16, 128)
     assert b.permuted_rows(cfg) == 16384 * 4 + 60 * 127 + (128 - (16384 * 4 + 60 * 127) % 128) % 128
     assert b.workspace_bytes(cfg, b.WS_LAYER) >= b.workspace_bytes(cfg, b.WS_PERMUTE) > 0
-    assert b.lib.c2r_route(C.byref(cfg), None, None, None, None, None, None, None) == -1
+    assert b.lib.c2r_route(C.byref(cfg), None, None, None, None, None, None, None, None) == -1
     bad = b.make_config(16, 60, 8, 16, 2, 1, 1, 0, b.BF16, 1)     # d % 8 != 0
     assert b.lib.c2r_gate_logits(C.byref(bad), None, None, None, None, None, None) == -2
     bad = b.make_config(16, 64, 65, 16, 2, 1, 1, 0, b.BF16, 1)    # E > 64
     assert b.lib.c2r_permuted_rows(C.byref(bad)) == -1
     bad = b.make_config(16, 64, 8, 16, 9, 1, 1, 0, b.BF16, 1)     # K > 8
-    assert b.lib.c2r_route(C.byref(bad), None, None, None, None, None, None, None) == -2
+    assert b.lib.c2r_route(C.byref(bad), None, None, None, None, None, None, None, None) == -2
 
 
 @pytest.mark.parametrize("E,P", [(8, 2), (16, 4), (60, 4), (60, 8), (7, 3), (5, 5), (9, 1)])
@@ -91,3 +91,11 @@ def test_bench_accounting_matches_the_workload_arithmetic():
     assert bench.flops_per_token(c2) == 3 * 6 * 4 * 4096 * 688
     # whole step at c3: 6.80 TFLOP, the figure the roofline line reports per 12 launches
     assert abs(bench.flops_per_token(c3) * c3.N / 1e12 - 6.803) < 1e-3
+    # bandwidth-bound calls at c3, bytes per token: dispatch reads a 4 KiB row and writes it K = 4 times
+    # (+ 64 B of index); the combine reads K + 1 rows (shared expert) and writes one -- in fp32 as stored
+    # (4 * 5 * 2048 + 4096 B) or in the storage type (2 * 6 * 2048 B)
+    moved, alg = bench.hbm_bytes(c3)
+    assert moved["permute"] == c3.N * (5 * 4096 + 64) and alg["permute"] == moved["permute"]
+    assert moved["combine"] == c3.N * (4 * 5 * 2048 + 4096) and alg["combine"] == c3.N * 2 * 6 * 2048
+    assert moved["spread_dY"] == c3.N * 5 * 4096
+    assert moved["gate_logits"] == c3.N * (4096 + 61 * 4) + 61 * 4096

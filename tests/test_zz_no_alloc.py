@@ -57,9 +57,39 @@ def test_static_scratch_permute_matches_workspace_permute_twice():
         assert int(got["counts"].sum()) == N * K
 
 
+@pytest.mark.parametrize("N", [150000, 559232])
+def test_static_scratch_large_batches_match_the_oracle(N):
+    """Index-only dispatch of batches past 1024 sort blocks (separate histogram / scan / rank launches),
+    the second one filling the built-in scratch to its last byte (4369 blocks * 60 experts * 4 B <= 1 MiB),
+    through both entry points, against the oracle."""
+    from oracle import c2r_oracle as O
+    from paper_2504_01337_b200 import binding as b
+    E, K, align = 60, 4, 128
+    rng = np.random.default_rng(N)
+    idx = np.argsort(-rng.standard_normal((N, E)).astype(np.float32), axis=1, kind="stable")[:, :K].astype(np.int32)
+    rank = rng.permutation(E).astype(np.int32)
+    cfg = b.make_config(N, 64, E, 16, K, K - 1, 1, 0, b.BF16, align)
+    assert b.workspace_bytes(cfg, b.WS_PERMUTE) <= (1 << 20)
+    ref = O.permute_index(idx, E, rank, align)
+    idx_d, rank_d = torch.from_numpy(idx).cuda(), torch.from_numpy(rank).cuda()
+    ws = torch.empty(b.workspace_bytes(cfg, b.WS_PERMUTE), dtype=torch.uint8, device="cuda")
+    for static in (False, True):
+        o = _outputs(b, cfg, E, K, N, 1, torch.bfloat16)
+        if static:
+            b.permute_static(cfg, idx_d, rank_d, None, o["counts"], o["offsets"], o["ros"], o["sor"], None, o["status"])
+        else:
+            b.permute(cfg, idx_d, rank_d, None, o["counts"], o["offsets"], o["ros"], o["sor"], None, o["status"], ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(o["counts"].cpu().numpy(), ref[0]) and np.array_equal(o["offsets"].cpu().numpy(), ref[1])
+        assert np.array_equal(o["ros"].cpu().numpy(), ref[2])
+        sor = o["sor"].cpu().numpy()
+        assert np.array_equal(sor[: ref[3].size], ref[3]) and np.all(sor[ref[3].size:] == -1)
+        assert int(o["status"].item()) == 0
+
+
 def test_static_scratch_limit_is_an_error_code():
     from paper_2504_01337_b200 import binding as b
-    # ceil(N*K/512) * E * 4 bytes = 4688 * 64 * 4 > 1 MiB: refused on the host, nothing is dereferenced
+    # ceil(N/128) * E * 4 bytes = 4688 * 64 * 4 > 1 MiB: refused on the host, nothing is dereferenced
     cfg = b.make_config(600000, 64, 64, 16, 4, 3, 1, 0, b.BF16, 1)
     t = torch.zeros(8, dtype=torch.int32, device="cuda")
     with pytest.raises(b.C2RError) as e:
