@@ -131,7 +131,7 @@ class ClockSampler:
                 "samples": len(sm), "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons)}
 
 
-def build_layer(wl, device, profile=True, keep=False, gather_fused=False):
+def build_layer(wl, device, profile=True, keep=False, gather_fused=False, fused_combine=False, side_stream=False):
     """Seeded synthetic layer of workload `wl` on `device`, routed with collaborator sets profiled
     from a calibration batch by the library itself (Eq. 2 / Eq. 4) and placed by co-activation.
     keep=True also returns the calibration state (device logits, routing, C, I_T, placement)."""
@@ -141,7 +141,7 @@ def build_layer(wl, device, profile=True, keep=False, gather_fused=False):
     from paper_2504_01337_b200.layer import C2RLayer, to_device
 
     lay = C2RLayer(wl.N, wl.d, wl.E, wl.I, wl.K, wl.T, wl.P, wl.I_s, wl.bf16, backward=True, profile=profile,
-                   device=device, gather_fused=gather_fused)
+                   device=device, gather_fused=gather_fused, fused_combine=fused_combine, side_stream=side_stream)
     Wg, wsg = G.gate_weights(wl)
     W1, W3, W2 = G.expert_weights(wl)
     lay.set_params(Wg, W1, W3, W2, wsg, G.shared_weights(wl))
@@ -186,50 +186,48 @@ def breakdown(lay, reps=3):
     nqs = B.swiglu_qparts(c, 1, c.I_s, c.N) if shared else 0
     qpart = torch.empty((max(nq, 1), R), dtype=torch.float32, device=t["X"].device)
     qspart = torch.empty((max(nqs, 1), c.N), dtype=torch.float32, device=t["X"].device)
-    row = dict(row_scale=t["w_row"], scale_kind=B.SCALE_ROW)
-    gate = dict(row_scale=t.get("z"), scale_kind=B.SCALE_SIGMOID)
-    calls = [
-        ("gate_logits", lambda: B.gate_logits(c, t["X"], t["Wg"], t.get("wsg"), t["L"], t.get("z"))),
+    fcomb = bool(c.flags & B.FLAG_FUSED_COMBINE)
+    sor = t["slot_of_row"] if (fused or fcomb) else None
+    o_fwd = B.expert_opts(t["w_row"], B.SCALE_ROW, X=t["X"] if fused else None, slot_of_row=sor, token_acc=t.get("Yacc"))
+    o_bwd = B.expert_opts(t["w_row"], B.SCALE_ROW, X=t["X"] if fused else None, slot_of_row=sor, token_acc=t.get("dXacc"),
+                          qpart=qpart)
+    o_sfwd = B.expert_opts(t.get("z"), B.SCALE_SIGMOID)
+    o_sbwd = B.expert_opts(t.get("z"), B.SCALE_SIGMOID, qpart=qspart)
+    calls = [("gate_logits", lambda: B.gate_logits(c, t["X"], t["Wg"], t.get("wsg"), t["L"], t.get("z")))]
+    if shared:
+        calls.append(("shared_fwd", lambda: B.grouped_swiglu_fwd(c, 1, c.I_s, c.N, t["X"], t["s_counts"], t["s_offsets"],
+                                                                 t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"],
+                                                                 t["Yacc"] if fcomb else t["Ys"], None, o_sfwd)))
+    elif fcomb:
+        calls.append(("zero_acc", lambda: (t["Yacc"].zero_(), t["dXacc"].zero_())))
+    calls += [
         ("route", lambda: B.route(c, t["L"], t.get("mask"), t["idx"], t["w"], None, t["status"], ws)),
         ("permute", lambda: B.permute(c, t["idx"], t.get("expert_rank"), None if fused else t["X"], t["counts"],
                                       t["offsets"], t["row_of_slot"], t["slot_of_row"], t.get("Xp"), t["status"], ws,
                                       t["w"], t["w_row"], True)),
-        ("swiglu_fwd", (lambda: B.grouped_swiglu_fwd_gather(c, c.E, c.I, R, t["X"], t["slot_of_row"], t["counts"],
-                                                            t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["Yp"],
-                                                            None, **row))
-         if fused else
-         (lambda: B.grouped_swiglu_fwd(c, c.E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"],
-                                       t["W2"], t["AB"], t["H"], t["Yp"], None, **row))),
-    ]
-    if shared:
-        calls.append(("shared_fwd", lambda: B.grouped_swiglu_fwd(c, 1, c.I_s, c.N, t["X"], t["s_counts"], t["s_offsets"],
-                                                                 t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["Ys"], None,
-                                                                 **gate)))
-    calls += [
-        ("combine", lambda: B.combine(c, t["Yp"], None, t["row_of_slot"], t.get("Ys"), None, t["Y"])),
+        ("swiglu_fwd", lambda: B.grouped_swiglu_fwd(c, c.E, c.I, R, t.get("Xp"), t["counts"], t["offsets"], t["W13p"],
+                                                    t["W2"], t["AB"], t["H"], t.get("Yp"), None, o_fwd)),
+        ("combine", lambda: B.combine(c, t.get("Yp"), None, t["row_of_slot"], t["Yacc"] if fcomb else t.get("Ys"), None,
+                                      t["Y"])),
         ("dispatch_volume", lambda: B.dispatch_volume(c, t["idx"], t["part"], t["volume"], t["volume"][4:],
                                                       t["volume"][4 + P * P:])),
-        ("spread_dY", lambda: B.permute_rows(c, t["dY"], t["row_of_slot"], t["counts"], t["offsets"], t["dYp"])),
-        ("swiglu_bwd", (lambda: B.grouped_swiglu_bwd_gather(c, c.E, c.I, R, t["X"], t["slot_of_row"], t["counts"],
-                                                            t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["dYp"],
-                                                            t["dAB"], t["dXp"], t["dW13p"], t["dW2"], False, None,
-                                                            qpart=qpart, **row))
-         if fused else
-         (lambda: B.grouped_swiglu_bwd(c, c.E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"],
-                                       t["W2"], t["AB"], t["H"], t["dYp"], t["dAB"], t["dXp"],
-                                       t["dW13p"], t["dW2"], False, None, qpart=qpart, **row))),
     ]
     if shared:
         calls.append(("shared_bwd", lambda: B.grouped_swiglu_bwd(c, 1, c.I_s, c.N, t["X"], t["s_counts"], t["s_offsets"],
                                                                  t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["dY"],
-                                                                 t["dABs"], t["dXs"], t["dWs13p"], t["dWs2"], False, None,
-                                                                 qpart=qspart, **gate)))
+                                                                 t["dABs"], t["dXacc"] if fcomb else t["dXs"], t["dWs13p"],
+                                                                 t["dWs2"], False, None, o_sbwd)))
     calls += [
+        ("spread_dY", lambda: B.permute_rows(c, t["dY"], t["row_of_slot"], t["counts"], t["offsets"], t["dYp"])),
+        ("swiglu_bwd", lambda: B.grouped_swiglu_bwd(c, c.E, c.I, R, t.get("Xp"), t["counts"], t["offsets"], t["W13p"],
+                                                    t["W2"], t["AB"], t["H"], t["dYp"], t["dAB"], t.get("dXp"),
+                                                    t["dW13p"], t["dW2"], False, None, o_bwd)),
         ("route_bwd", lambda: B.route_bwd_scaled(c, t["w"], t["row_of_slot"], qpart, nq, t.get("z"), qspart, nqs,
                                                  t["dw"], t["dl"], t.get("dz"))),
         ("gate_bwd", lambda: B.gate_bwd(c, t["X"], t.get("Xp"), t["counts"], t["offsets"], t["slot_of_row"], t["dl"],
                                         t.get("dz"), t["dWg"], t.get("dwsg"), ws)),
-        ("unpermute_grad", lambda: B.unpermute_grad(c, t["dXp"], t["row_of_slot"], t.get("dXs"), t["idx"], t["dl"],
+        ("unpermute_grad", lambda: B.unpermute_grad(c, t.get("dXp"), t["row_of_slot"],
+                                                    t["dXacc"] if fcomb else t.get("dXs"), t["idx"], t["dl"],
                                                     t["Wg"], t.get("dz"), t.get("wsg"), t["dX"])),
         ("collab_count", lambda: B.collab_count(c, t["idx"], c.N, t["C"])),
         ("collab_sets", lambda: B.collab_sets(c, t["C"], t["I_T"], t["mask_next"])),
@@ -428,13 +426,18 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c3s", "c5"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c3s", "c3e", "c5"])
     ap.add_argument("--impl", default="c2r", choices=["c2r", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=128)
     ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
     ap.add_argument("--no-reports", action="store_true", help="skip the Top-K vs C2R dispatch reports")
+    ap.add_argument("--combine", default="gather", choices=["gather", "fused"],
+                    help="gather: the GEMMs store fp32 partials and a gather pass sums them (deterministic); fused: the GEMM "
+                         "epilogues add their rows into per-token fp32 accumulators (order of the adds not fixed)")
+    ap.add_argument("--streams", type=int, default=2, choices=[1, 2],
+                    help="2: the shared expert's GEMMs run on a second stream beside the routing chain")
     ap.add_argument("--dispatch", default="permute", choices=["permute", "gather-fused"],
                     help="permute: c2r_permute writes Xp (faster); gather-fused: the expert GEMMs read token rows from X, no permuted copy")
     args = ap.parse_args()
@@ -459,7 +462,8 @@ def main():
     # every rank is an independent data-parallel replica: same parameters, its own batch
     wl_rank = RP.rank_workload(wl, rank)
     fused = args.dispatch == "gather-fused" and wl.bf16
-    lay, cal = build_layer(wl, device, keep=True, gather_fused=fused)
+    fcomb = args.combine == "fused"
+    lay, cal = build_layer(wl, device, keep=True, gather_fused=fused, fused_combine=fcomb, side_stream=args.streams == 2)
     if args.workload == "c5":
         # large-batch training step: the sets refreshed from this step's routing (Eq. 2, Eq. 4) are the
         # ones the next step routes with (the refresh is the last thing a step enqueues)
@@ -564,6 +568,7 @@ def main():
             "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "E": wl.E, "I": wl.I, "K": wl.K, "T": wl.T,
                        "P": wl.P, "I_s": wl.I_s, "row_align": lay.cfg.row_align, "parallelism": f"dp{world} (replicas)",
                        "step": "fwd+bwd+collab refresh (c2r_train_step)", "dispatch": "gather-fused" if fused else "permute",
+                       "combine": args.combine, "streams": args.streams if wl.I_s else 1,
                        "l2": "working set (>1 GB weights + activations) exceeds the 126 MB L2"},
             "clocks": clocks,
             "e2e": {"value": RP.whole_job_rate(wl.N, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": 2 * nbytes,

@@ -66,8 +66,11 @@ typedef struct c2r_config {
 
 /* c2r_config.flags */
 enum {
-  C2R_FLAG_GATHER_FUSED = 1 /* layer drivers (bf16 tensor-core path): the expert GEMMs fetch token rows straight
-                               from X through slot_of_row (TMA row gather); Xp is neither written nor read */
+  C2R_FLAG_GATHER_FUSED = 1,  /* layer drivers (bf16 tensor-core path): the expert GEMMs fetch token rows straight
+                                 from X through slot_of_row (TMA row gather); Xp is neither written nor read */
+  C2R_FLAG_FUSED_COMBINE = 2  /* layer drivers: the down-projection and the dXp GEMM add their rows straight into
+                                 per-token fp32 accumulators (Yacc, dXacc) instead of storing Yp / dXp for a gather
+                                 pass; order of the fp32 adds not fixed (see c2r_expert_opts.token_acc) */
 };
 
 enum { C2R_WS_PERMUTE = 0, C2R_WS_GATE_BWD = 1, C2R_WS_LAYER = 2, C2R_WS_DISPATCH_DEDUP = 3 };
@@ -210,11 +213,34 @@ int c2r_pack_weights(const c2r_config* cfg, int n_experts, int I, const void* W1
 int c2r_unpack_weights(const c2r_config* cfg, int n_experts, int I, const void* W13p, void* W1,
                        void* W3, void* stream);
 
+/* Options of the two grouped SwiGLU calls below (a NULL pointer to it, or a zeroed struct, selects none).
+ *   row_scale / scale_kind: per-row scale s_r of H (C2R_SCALE_*; row_scale [R] float).  With the Eq. 1
+ *     weights as row scale, Yp already carries the weight of Sec. 3.1's weighted sum.
+ *   X with slot_of_row: the dispatch folded into the GEMMs (the gather-fused form): wherever the calls read
+ *     row r of Xp, the kernels read row slot_of_row[r] / K of X [N,d] T instead (zeros where slot_of_row[r] < 0),
+ *     so c2r_permute can run with X == NULL and no permuted copy of the hidden states exists (Xp may be NULL).
+ *     Same results, bit for bit.  bf16 tensor-core shapes only, else C2R_ERR_UNSUPPORTED_SHAPE.
+ *   token_acc with slot_of_row: the combine folded into the GEMM epilogue: the [R,d] float result (Yp forward,
+ *     dXp backward) is not stored; row r is added into token_acc[slot_of_row[r] / K, :] ([N,d] float, which the
+ *     caller has zeroed or pre-loaded, e.g. with the shared expert's output).  The adds are fp32 atomics: the
+ *     order in which a token's K contributions arrive is not fixed, so results may differ in the last bits
+ *     from run to run.  Yp / dXp may then be NULL.
+ *   qpart (backward only): [c2r_swiglu_qparts(...)][R] float, partial sums whose total over the first index is
+ *     q_r = <dH'_r, H_r> = s_r dLoss/ds_r, the gradient w.r.t. the row's scale times the scale (added up in
+ *     index order by c2r_route_bwd_scaled); rows outside every expert's segment are not written. */
+typedef struct c2r_expert_opts {
+  const float* row_scale;
+  int32_t scale_kind;
+  int32_t reserved;
+  const void* X;
+  const int32_t* slot_of_row;
+  float* token_acc;
+  float* qpart;
+} c2r_expert_opts;
+
 /* Sec. 3.1: expert evaluation of the routed tokens; expert = SwiGLU MLP without biases.
  * For each expert e on rows [offsets[e], offsets[e]+counts[e]) of Xp:
- *   A = Xp W1_e^T, B = Xp W3_e^T, H = s_r silu(A) * B, Yp = H W2_e^T,
- * s_r the optional per-row scale (C2R_SCALE_*; row_scale [R] float, NULL with C2R_SCALE_NONE).  With the
- * Eq. 1 weights as row scale, Yp already carries the weight of Sec. 3.1's weighted sum.
+ *   A = Xp W1_e^T, B = Xp W3_e^T, H = s_r silu(A) * B, Yp = H W2_e^T      (s_r = 1 without a row scale).
  * Xp [R,d] T; counts [n_experts], offsets [n_experts+1] int32 (device); W13p packed (above);
  * W2 [n_experts, d, I] T.  out: AB [R, 2I] T (what the backward pass needs from A and B, in the
  * packed column layout: the local derivatives B silu'(A) in the gate columns and silu(A) in the up
@@ -227,46 +253,26 @@ int c2r_unpack_weights(const c2r_config* cfg, int n_experts, int I, const void* 
  * receives C2R_STATUS_WAIT_TIMEOUT if a bounded wait inside the kernel gave up (results invalid). */
 int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                            const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
-                           const float* row_scale, int scale_kind, void* AB, void* H, void* Yp, int32_t* status,
-                           void* stream);
+                           void* AB, void* H, void* Yp, const c2r_expert_opts* opts, int32_t* status, void* stream);
 
 /* Backward of the above, given dYp = dLoss/dYp:  dH' = dYp W2 (the gradient w.r.t. the scaled H);
  * dA = s_r dH' B silu'(A); dB = s_r dH' silu(A); dXp = dA W1 + dB W3; dW2_e = dYp^T H; dW1_e = dA^T Xp;
  * dW3_e = dB^T Xp.  dYp [R,d] T (padding rows zero); AB, H as the forward call wrote them;
  * out: dAB [R,2I] T (packed columns), dXp [R,d] float, dW13p [n_experts,2I,d] T (packed rows),
- * dW2 [n_experts,d,I] T.  accumulate != 0 adds into the weight gradients.
- * qpart (optional) [c2r_swiglu_qparts(...)][R] float: partial sums whose total over the first index is
- * q_r = <dH'_r, H_r> = s_r dLoss/ds_r, the gradient w.r.t. the row's scale times the scale (added up in index
- * order by c2r_route_bwd_scaled); rows outside every expert's segment are not written. */
+ * dW2 [n_experts,d,I] T.  accumulate != 0 adds into the weight gradients. */
 int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                            const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
-                           const void* AB, const void* H, const void* dYp, const float* row_scale, int scale_kind,
-                           void* dAB, void* dXp, void* dW13p, void* dW2, float* qpart, int accumulate,
-                           int32_t* status, void* stream);
+                           const void* AB, const void* H, const void* dYp, void* dAB, void* dXp, void* dW13p,
+                           void* dW2, int accumulate, const c2r_expert_opts* opts, int32_t* status, void* stream);
 
-/* First dimension of qpart for this shape (host function; -1 on a bad argument). */
+/* First dimension of c2r_expert_opts.qpart for this shape (host function; -1 on a bad argument). */
 int c2r_swiglu_qparts(const c2r_config* cfg, int n_experts, int I, int64_t R);
-
-/* The two calls above with the dispatch folded into the GEMMs (an addition of this library: the gather-fused
- * form of the dispatch): wherever they read row r of Xp, the kernels read row slot_of_row[r] / K of X
- * instead (zeros where slot_of_row[r] < 0), so c2r_permute can be called with X == NULL and no permuted copy
- * of the hidden states exists.  Same outputs, bit for bit.  bf16 tensor-core shapes only (d % 16 == 0,
- * I % 16 == 0, row_align a multiple of 128): anything else returns C2R_ERR_UNSUPPORTED_SHAPE.
- * X [N,d] T; slot_of_row [R] int32 as c2r_permute wrote it. */
-int c2r_grouped_swiglu_fwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
-                                  const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
-                                  const void* W13p, const void* W2, const float* row_scale, int scale_kind, void* AB,
-                                  void* H, void* Yp, int32_t* status, void* stream);
-int c2r_grouped_swiglu_bwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
-                                  const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
-                                  const void* W13p, const void* W2, const void* AB, const void* H, const void* dYp,
-                                  const float* row_scale, int scale_kind, void* dAB, void* dXp, void* dW13p, void* dW2,
-                                  float* qpart, int accumulate, int32_t* status, void* stream);
 
 /* Sec. 3.1 (weighted sum of the selected experts' outputs):
  * Y[t,:] = sum_k w[t,k] * Yp[row_of_slot[t*K+k],:]  (k ascending, fp32)
  *          + sigmoid(z[t]) * Ys[t,:] when Ys != NULL (gated shared expert).
  * w == NULL / z == NULL: that factor is 1 (the expert call already applied it as its row scale).
+ * Yp == NULL: no such term (the GEMMs already added their rows into Ys: Y is Ys in the storage type).
  * Yp [R,d] float; Ys [N,d] float; out: Y [N,d] T. */
 int c2r_combine(const c2r_config* cfg, const void* Yp, const float* w, const int32_t* row_of_slot,
                 const void* Ys, const float* z, void* Y, void* stream);
@@ -307,7 +313,8 @@ int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp, const int
  * dX[t,:] = sum_k dXp[row_of_slot[t*K+k],:]  + dXs[t,:]                (shared expert, optional)
  *           + sum_k dl[t,k] Wg[idx[t,k],:] + dz[t] wsg[:]              (gate, optional)
  *           + dX[t,:] when accumulate != 0.
- * dXp [R,d] float; dXs [N,d] float; out: dX [N,d] T. */
+ * dXp [R,d] float (NULL: no such term, e.g. when the GEMMs already added their rows into dXs);
+ * dXs [N,d] float; out: dX [N,d] T. */
 int c2r_unpermute_grad(const c2r_config* cfg, const void* dXp, const int32_t* row_of_slot, const void* dXs,
                        const int32_t* idx, const float* dl, const void* Wg, const float* dz, const void* wsg,
                        void* dX, int accumulate, void* stream);
@@ -356,6 +363,7 @@ typedef struct c2r_layer_buffers {
   int32_t* s_counts;    /* [1]  = {N}   (device) */
   int32_t* s_offsets;   /* [2]  = {0,N} (device) */
   void* Y;              /* [N,d] T: layer output */
+  float* Yacc;          /* [N,d] float, only with C2R_FLAG_FUSED_COMBINE (Yp, Ys may then be NULL) */
   uint64_t* volume;     /* [4 + 2*P*P] totals, send_naive, send_dedup */
   int32_t* status;      /* one int32 */
   /* backward */
@@ -375,6 +383,7 @@ typedef struct c2r_layer_buffers {
   float* dWg;     /* [E,d] */
   float* dwsg;    /* [d] */
   void* dX;       /* [N,d] T */
+  float* dXacc;   /* [N,d] float, only with C2R_FLAG_FUSED_COMBINE (dXp, dXs may then be NULL) */
   /* live profiling (c2r_train_step) */
   int32_t* C;          /* [E,E] */
   int32_t* I_T;        /* [E,T] */

@@ -40,9 +40,9 @@ class Config(C.Structure):
 _LAYER_FIELDS = [
     "X", "Wg", "wsg", "W13p", "W2", "Ws13p", "Ws2", "mask", "expert_rank", "part",
     "L", "z", "idx", "w", "counts", "offsets", "row_of_slot", "slot_of_row", "w_row", "Xp", "AB", "H", "Yp",
-    "ABs", "Hs", "Ys", "s_counts", "s_offsets", "Y", "volume", "status",
+    "ABs", "Hs", "Ys", "s_counts", "s_offsets", "Y", "Yacc", "volume", "status",
     "dY", "dYp", "dAB", "dXp", "dABs", "dXs", "dw", "dl", "dz",
-    "dW13p", "dW2", "dWs13p", "dWs2", "dWg", "dwsg", "dX",
+    "dW13p", "dW2", "dWs13p", "dWs2", "dWg", "dwsg", "dX", "dXacc",
     "C", "I_T", "mask_next", "stream2", "ev_fork", "ev_join", "ws",
 ]
 
@@ -51,14 +51,18 @@ class LayerBuffers(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in _LAYER_FIELDS] + [("ws_bytes", C.c_size_t)]
 
 
+class ExpertOpts(C.Structure):
+    _fields_ = [("row_scale", C.c_void_p), ("scale_kind", C.c_int32), ("reserved", C.c_int32), ("X", C.c_void_p),
+                ("slot_of_row", C.c_void_p), ("token_acc", C.c_void_p), ("qpart", C.c_void_p)]
+
+
 EXPORTS = [
     "c2r_workspace_bytes", "c2r_permuted_rows", "c2r_last_cuda_error", "c2r_launch_count", "c2r_gate_logits", "c2r_route",
     "c2r_collab_count", "c2r_collab_sets", "c2r_collab_degree", "c2r_place_experts", "c2r_permute", "c2r_pack_weights",
     "c2r_unpack_weights", "c2r_grouped_swiglu_fwd", "c2r_grouped_swiglu_bwd", "c2r_combine", "c2r_combine_bwd",
     "c2r_route_bwd", "c2r_gate_bwd", "c2r_unpermute_grad", "c2r_dispatch_volume", "c2r_layer_fwd",
     "c2r_layer_bwd", "c2r_train_step", "c2r_permute_static", "c2r_dispatch_dedup",
-    "c2r_grouped_swiglu_fwd_gather", "c2r_grouped_swiglu_bwd_gather", "c2r_permute_rows", "c2r_swiglu_qparts",
-    "c2r_route_bwd_scaled",
+    "c2r_permute_rows", "c2r_swiglu_qparts", "c2r_route_bwd_scaled",
 ]
 
 _P = C.c_void_p
@@ -84,10 +88,8 @@ _SIGS = {
     "c2r_dispatch_dedup": [_CFG] + [_P] * 16 + [C.c_size_t, _P],
     "c2r_pack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
     "c2r_unpack_weights": [_CFG, C.c_int, C.c_int, _P, _P, _P, _P],
-    "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 6 + [C.c_int] + [_P] * 5,
-    "c2r_grouped_swiglu_bwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 9 + [C.c_int] + [_P] * 5 + [C.c_int, _P, _P],
-    "c2r_grouped_swiglu_fwd_gather": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 7 + [C.c_int] + [_P] * 5,
-    "c2r_grouped_swiglu_bwd_gather": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 10 + [C.c_int] + [_P] * 5 + [C.c_int, _P, _P],
+    "c2r_grouped_swiglu_fwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 8 + [C.POINTER(ExpertOpts), _P, _P],
+    "c2r_grouped_swiglu_bwd": [_CFG, C.c_int, C.c_int, C.c_int64] + [_P] * 12 + [C.c_int, C.POINTER(ExpertOpts), _P, _P],
     "c2r_combine": [_CFG] + [_P] * 7,
     "c2r_combine_bwd": [_CFG] + [_P] * 12,
     "c2r_route_bwd": [_CFG] + [_P] * 4,
@@ -104,6 +106,7 @@ for _name, _sig in _SIGS.items():
 
 
 FLAG_GATHER_FUSED = 1
+FLAG_FUSED_COMBINE = 2
 SCALE_NONE, SCALE_ROW, SCALE_SIGMOID = 0, 1, 2
 
 
@@ -220,37 +223,26 @@ def unpack_weights(cfg, n_experts, I, W13p, W1, W3):
     _call("c2r_unpack_weights", C.byref(cfg), n_experts, I, _ptr(W13p), _ptr(W1), _ptr(W3), _stream())
 
 
-def _scale_kind(row_scale, scale_kind):
-    return SCALE_NONE if row_scale is None else int(scale_kind)
+def expert_opts(row_scale=None, scale_kind=SCALE_ROW, X=None, slot_of_row=None, token_acc=None, qpart=None):
+    """c2r_expert_opts from tensors (None members stay NULL)."""
+    o = ExpertOpts()
+    o.row_scale = _ptr(row_scale)
+    o.scale_kind = SCALE_NONE if row_scale is None else int(scale_kind)
+    o.X, o.slot_of_row, o.token_acc, o.qpart = _ptr(X), _ptr(slot_of_row), _ptr(token_acc), _ptr(qpart)
+    return o
 
 
-def grouped_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, status=None, row_scale=None,
-                       scale_kind=SCALE_ROW):
+def grouped_swiglu_fwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, Yp, status=None, opts=None):
     _call("c2r_grouped_swiglu_fwd", C.byref(cfg), n_experts, I, int(R), _ptr(Xp), _ptr(counts), _ptr(offsets),
-          _ptr(W13p), _ptr(W2), _ptr(row_scale), _scale_kind(row_scale, scale_kind), _ptr(AB), _ptr(H), _ptr(Yp),
-          _ptr(status), _stream())
+          _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(Yp), None if opts is None else C.byref(opts), _ptr(status),
+          _stream())
 
 
 def grouped_swiglu_bwd(cfg, n_experts, I, R, Xp, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p, dW2,
-                       accumulate=False, status=None, row_scale=None, scale_kind=SCALE_ROW, qpart=None):
+                       accumulate=False, status=None, opts=None):
     _call("c2r_grouped_swiglu_bwd", C.byref(cfg), n_experts, I, int(R), _ptr(Xp), _ptr(counts), _ptr(offsets),
-          _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(row_scale), _scale_kind(row_scale, scale_kind),
-          _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2), _ptr(qpart), int(accumulate), _ptr(status), _stream())
-
-
-def grouped_swiglu_fwd_gather(cfg, n_experts, I, R, X, slot_of_row, counts, offsets, W13p, W2, AB, H, Yp, status=None,
-                              row_scale=None, scale_kind=SCALE_ROW):
-    _call("c2r_grouped_swiglu_fwd_gather", C.byref(cfg), n_experts, I, int(R), _ptr(X), _ptr(slot_of_row), _ptr(counts),
-          _ptr(offsets), _ptr(W13p), _ptr(W2), _ptr(row_scale), _scale_kind(row_scale, scale_kind), _ptr(AB), _ptr(H),
-          _ptr(Yp), _ptr(status), _stream())
-
-
-def grouped_swiglu_bwd_gather(cfg, n_experts, I, R, X, slot_of_row, counts, offsets, W13p, W2, AB, H, dYp, dAB, dXp, dW13p,
-                              dW2, accumulate=False, status=None, row_scale=None, scale_kind=SCALE_ROW, qpart=None):
-    _call("c2r_grouped_swiglu_bwd_gather", C.byref(cfg), n_experts, I, int(R), _ptr(X), _ptr(slot_of_row), _ptr(counts),
-          _ptr(offsets), _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(row_scale),
-          _scale_kind(row_scale, scale_kind), _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2), _ptr(qpart), int(accumulate),
-          _ptr(status), _stream())
+          _ptr(W13p), _ptr(W2), _ptr(AB), _ptr(H), _ptr(dYp), _ptr(dAB), _ptr(dXp), _ptr(dW13p), _ptr(dW2),
+          int(accumulate), None if opts is None else C.byref(opts), _ptr(status), _stream())
 
 
 def combine(cfg, Yp, w, row_of_slot, Ys, z, Y):

@@ -71,10 +71,19 @@ static int check_gemm_args(const c2r_config* cfg, int nE, int I, int64_t R) {
   return C2R_OK;
 }
 
-static int check_scale(const float* row_scale, int scale_kind) {
-  C2R_REQUIRE(scale_kind == C2R_SCALE_NONE || scale_kind == C2R_SCALE_ROW || scale_kind == C2R_SCALE_SIGMOID,
+// Validates the options and copies them into the call.
+static int apply_opts(const c2r_config* cfg, const c2r_expert_opts* o, SwigluCall& a, bool backward) {
+  if (o == nullptr) return C2R_OK;
+  C2R_REQUIRE(o->scale_kind == C2R_SCALE_NONE || o->scale_kind == C2R_SCALE_ROW || o->scale_kind == C2R_SCALE_SIGMOID,
               C2R_ERR_INVALID_ARG);
-  C2R_REQUIRE(scale_kind == C2R_SCALE_NONE || row_scale != nullptr, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(o->scale_kind == C2R_SCALE_NONE || o->row_scale != nullptr, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE((!o->X && !o->token_acc) || o->slot_of_row, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(backward || !o->qpart, C2R_ERR_INVALID_ARG);
+  a.row_scale = o->row_scale; a.scale_kind = o->scale_kind;
+  a.X = o->X; a.slot_of_row = o->slot_of_row; a.token_acc = o->token_acc; a.qpart = o->qpart;
+  if (a.X != nullptr)  // the row gather exists on the tensor-core path only
+    C2R_REQUIRE(tc_supported(cfg, a.nE, a.I, a.R) && (((uintptr_t)a.X) & 15u) == 0, C2R_ERR_UNSUPPORTED_SHAPE);
+  if (a.token_acc != nullptr) C2R_REQUIRE((((uintptr_t)a.token_acc) & 15u) == 0, C2R_ERR_INVALID_ARG);
   return C2R_OK;
 }
 
@@ -99,72 +108,34 @@ extern "C" int c2r_swiglu_qparts(const c2r_config* cfg, int n_experts, int I, in
 
 extern "C" int c2r_grouped_swiglu_fwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                                       const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
-                                      const float* row_scale, int scale_kind, void* AB, void* H, void* Yp,
-                                      int32_t* status, void* stream) {
+                                      void* AB, void* H, void* Yp, const c2r_expert_opts* opts, int32_t* status,
+                                      void* stream) {
   int rc = check_gemm_args(cfg, n_experts, I, R);
   if (rc) return rc;
-  C2R_REQUIRE(Xp && counts && offsets && W13p && W2 && H && Yp, C2R_ERR_INVALID_ARG);
-  if ((rc = check_scale(row_scale, scale_kind))) return rc;
   SwigluCall a{};
   a.nE = n_experts; a.I = I; a.R = R; a.Xp = Xp; a.counts = counts; a.offsets = offsets; a.W13p = W13p; a.W2 = W2;
-  a.row_scale = row_scale; a.scale_kind = scale_kind; a.AB = AB; a.H = H; a.Yp = Yp; a.status = status;
+  a.AB = AB; a.H = H; a.Yp = Yp; a.status = status;
+  if ((rc = apply_opts(cfg, opts, a, false))) return rc;
+  C2R_REQUIRE((Xp || a.X) && counts && offsets && W13p && W2 && H && (Yp || a.token_acc), C2R_ERR_INVALID_ARG);
   return swiglu_fwd_dispatch(cfg, a, as_stream(stream));
 }
 
 extern "C" int c2r_grouped_swiglu_bwd(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* Xp,
                                       const int32_t* counts, const int32_t* offsets, const void* W13p, const void* W2,
-                                      const void* AB, const void* H, const void* dYp, const float* row_scale,
-                                      int scale_kind, void* dAB, void* dXp, void* dW13p, void* dW2, float* qpart,
-                                      int accumulate, int32_t* status, void* stream) {
+                                      const void* AB, const void* H, const void* dYp, void* dAB, void* dXp,
+                                      void* dW13p, void* dW2, int accumulate, const c2r_expert_opts* opts,
+                                      int32_t* status, void* stream) {
   int rc = check_gemm_args(cfg, n_experts, I, R);
   if (rc) return rc;
-  C2R_REQUIRE(Xp && counts && offsets && W13p && W2 && AB && H && dYp && dAB && dXp && dW13p && dW2,
-              C2R_ERR_INVALID_ARG);
-  if ((rc = check_scale(row_scale, scale_kind))) return rc;
   SwigluCall a{};
   a.nE = n_experts; a.I = I; a.R = R; a.Xp = Xp; a.counts = counts; a.offsets = offsets; a.W13p = W13p; a.W2 = W2;
-  a.row_scale = row_scale; a.scale_kind = scale_kind; a.AB = const_cast<void*>(AB); a.H = const_cast<void*>(H);
-  a.dYp = dYp; a.dAB = dAB; a.dXp = dXp; a.dW13p = dW13p; a.dW2 = dW2; a.qpart = qpart; a.accumulate = accumulate;
-  a.status = status;
-  return swiglu_bwd_dispatch(cfg, a, as_stream(stream));
-}
-
-extern "C" int c2r_grouped_swiglu_fwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
-                                             const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
-                                             const void* W13p, const void* W2, const float* row_scale, int scale_kind,
-                                             void* AB, void* H, void* Yp, int32_t* status, void* stream) {
-  int rc = check_gemm_args(cfg, n_experts, I, R);
-  if (rc) return rc;
-  C2R_REQUIRE(X && slot_of_row && counts && offsets && W13p && W2 && H && Yp, C2R_ERR_INVALID_ARG);
-  if ((rc = check_scale(row_scale, scale_kind))) return rc;
-  C2R_REQUIRE(tc_supported(cfg, n_experts, I, R) && (((uintptr_t)X) & 15u) == 0, C2R_ERR_UNSUPPORTED_SHAPE);
-  if (R == 0) return C2R_OK;
-  SwigluCall a{};
-  a.nE = n_experts; a.I = I; a.R = R; a.counts = counts; a.offsets = offsets; a.W13p = W13p; a.W2 = W2;
-  a.row_scale = row_scale; a.scale_kind = scale_kind; a.AB = AB; a.H = H; a.Yp = Yp; a.status = status;
-  a.X = X; a.slot_of_row = slot_of_row;
-  return tc_swiglu_fwd(cfg, a, as_stream(stream));
-}
-
-extern "C" int c2r_grouped_swiglu_bwd_gather(const c2r_config* cfg, int n_experts, int I, int64_t R, const void* X,
-                                             const int32_t* slot_of_row, const int32_t* counts, const int32_t* offsets,
-                                             const void* W13p, const void* W2, const void* AB, const void* H,
-                                             const void* dYp, const float* row_scale, int scale_kind, void* dAB,
-                                             void* dXp, void* dW13p, void* dW2, float* qpart, int accumulate,
-                                             int32_t* status, void* stream) {
-  int rc = check_gemm_args(cfg, n_experts, I, R);
-  if (rc) return rc;
-  C2R_REQUIRE(X && slot_of_row && counts && offsets && W13p && W2 && AB && H && dYp && dAB && dXp && dW13p && dW2,
+  a.AB = const_cast<void*>(AB); a.H = const_cast<void*>(H); a.dYp = dYp; a.dAB = dAB; a.dXp = dXp; a.dW13p = dW13p;
+  a.dW2 = dW2; a.accumulate = accumulate; a.status = status;
+  if ((rc = apply_opts(cfg, opts, a, true))) return rc;
+  C2R_REQUIRE((Xp || a.X) && counts && offsets && W13p && W2 && AB && H && dYp && dAB && (dXp || a.token_acc) && dW13p &&
+                  dW2,
               C2R_ERR_INVALID_ARG);
-  if ((rc = check_scale(row_scale, scale_kind))) return rc;
-  C2R_REQUIRE(tc_supported(cfg, n_experts, I, R) && (((uintptr_t)X) & 15u) == 0, C2R_ERR_UNSUPPORTED_SHAPE);
-  if (R == 0) return C2R_OK;
-  SwigluCall a{};
-  a.nE = n_experts; a.I = I; a.R = R; a.counts = counts; a.offsets = offsets; a.W13p = W13p; a.W2 = W2;
-  a.row_scale = row_scale; a.scale_kind = scale_kind; a.AB = const_cast<void*>(AB); a.H = const_cast<void*>(H);
-  a.dYp = dYp; a.dAB = dAB; a.dXp = dXp; a.dW13p = dW13p; a.dW2 = dW2; a.qpart = qpart; a.accumulate = accumulate;
-  a.status = status; a.X = X; a.slot_of_row = slot_of_row;
-  return tc_swiglu_bwd(cfg, a, as_stream(stream));
+  return swiglu_bwd_dispatch(cfg, a, as_stream(stream));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -230,42 +201,56 @@ struct SideStream {
   }
 };
 
+// The fused combine needs the fp32 per-token accumulators.
+static bool fused_combine(const c2r_config* cfg) { return (cfg->flags & C2R_FLAG_FUSED_COMBINE) != 0; }
+
 extern "C" int c2r_layer_fwd(const c2r_config* cfg, const c2r_layer_buffers* b, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   C2R_REQUIRE(b, C2R_ERR_INVALID_ARG);
   const bool shared = cfg->I_s > 0;
+  const bool fcomb = fused_combine(cfg);
   C2R_REQUIRE(b->ws && b->ws_bytes >= c2r_workspace_bytes(cfg, C2R_WS_LAYER), C2R_ERR_WORKSPACE);
-  C2R_REQUIRE(b->w_row, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE(b->w_row && (fcomb ? b->Yacc != nullptr : b->Yp != nullptr), C2R_ERR_INVALID_ARG);
   if (shared)
-    C2R_REQUIRE(b->wsg && b->z && b->Ws13p && b->Ws2 && b->Hs && b->Ys && b->s_counts && b->s_offsets,
+    C2R_REQUIRE(b->wsg && b->z && b->Ws13p && b->Ws2 && b->Hs && (fcomb || b->Ys) && b->s_counts && b->s_offsets,
                 C2R_ERR_INVALID_ARG);
   const int64_t R = permuted_rows(cfg);
   const LayerWs ws = layer_ws(cfg, b->ws);
   const SideStream ss(b, stream, shared);
   C2R_TRY(gate_logits_impl(cfg, b->X, b->Wg, shared ? b->wsg : nullptr, b->L, b->z, b->status, stream));
   if (shared) {
-    // shared expert, its sigmoid gate applied to H inside the GEMM: Ys = sigmoid(z) * Shared(x)
+    // shared expert, its sigmoid gate applied to H inside the GEMM: Ys = sigmoid(z) * Shared(x).  With the fused
+    // combine its output initialises the per-token accumulator the routed experts then add to.
+    c2r_expert_opts o{};
+    o.row_scale = b->z; o.scale_kind = C2R_SCALE_SIGMOID;
     C2R_TRY(ss.fork());
-    C2R_TRY(c2r_grouped_swiglu_fwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->z,
-                                   C2R_SCALE_SIGMOID, b->ABs, b->Hs, b->Ys, b->status, ss.work()));
+    C2R_TRY(c2r_grouped_swiglu_fwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
+                                   b->Hs, fcomb ? (void*)b->Yacc : b->Ys, &o, b->status, ss.work()));
+  } else if (fcomb) {
+    C2R_CUDA(cudaMemsetAsync(b->Yacc, 0, sizeof(float) * (size_t)cfg->N * cfg->d, as_stream(stream)));
   }
   // routing leaves the dispatch's per-block histogram in the workspace; the dispatch also spreads the weights
   C2R_TRY(route_impl(cfg, b->L, b->mask, b->idx, b->w, nullptr, b->status, (int32_t*)ws.permute, stream));
-  const bool fused = gather_fused(cfg, b->X);
-  C2R_TRY(permute_call(cfg, b->idx, b->expert_rank, fused ? nullptr : b->X, b->counts, b->offsets, b->row_of_slot,
+  const bool gfused = gather_fused(cfg, b->X);
+  C2R_TRY(permute_call(cfg, b->idx, b->expert_rank, gfused ? nullptr : b->X, b->counts, b->offsets, b->row_of_slot,
                        b->slot_of_row, b->Xp, b->status, ws.permute, align256(permute_ws_bytes(cfg)), stream, cfg->N > 0,
                        b->w, b->w_row));
   // routed experts with the Eq. 1 weight of each row applied to H: Yp = w * Expert(x)
-  if (fused)
-    C2R_TRY(c2r_grouped_swiglu_fwd_gather(cfg, cfg->E, cfg->I, R, b->X, b->slot_of_row, b->counts, b->offsets, b->W13p,
-                                          b->W2, b->w_row, C2R_SCALE_ROW, b->AB, b->H, b->Yp, b->status, stream));
-  else
-    C2R_TRY(c2r_grouped_swiglu_fwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->w_row,
-                                   C2R_SCALE_ROW, b->AB, b->H, b->Yp, b->status, stream));
-  C2R_TRY(ss.join());
+  c2r_expert_opts o{};
+  o.row_scale = b->w_row; o.scale_kind = C2R_SCALE_ROW;
+  if (gfused) { o.X = b->X; o.slot_of_row = b->slot_of_row; }
+  if (fcomb) {
+    o.token_acc = b->Yacc; o.slot_of_row = b->slot_of_row;
+    C2R_TRY(ss.join());  // the accumulator holds the shared expert's term before the routed rows are added
+  }
+  C2R_TRY(c2r_grouped_swiglu_fwd(cfg, cfg->E, cfg->I, R, gfused ? nullptr : b->Xp, b->counts, b->offsets, b->W13p, b->W2,
+                                 b->AB, b->H, fcomb ? nullptr : b->Yp, &o, b->status, stream));
+  if (!fcomb) C2R_TRY(ss.join());
   // the weights are already inside Yp and Ys: a plain sum over the token's K rows plus the shared term
-  C2R_TRY(c2r_combine(cfg, b->Yp, nullptr, b->row_of_slot, shared ? b->Ys : nullptr, nullptr, b->Y, stream));
+  // (fused combine: the sum is complete, what is left is the conversion to the storage type)
+  C2R_TRY(c2r_combine(cfg, fcomb ? nullptr : b->Yp, nullptr, b->row_of_slot,
+                      fcomb ? (void*)b->Yacc : (shared ? b->Ys : nullptr), nullptr, b->Y, stream));
   if (b->part && b->volume) {
     const int P = cfg->P;
     C2R_TRY(c2r_dispatch_volume(cfg, b->idx, b->part, b->volume, b->volume + 4, b->volume + 4 + P * P, stream));
@@ -278,37 +263,47 @@ extern "C" int c2r_layer_bwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
   if (rc) return rc;
   C2R_REQUIRE(b, C2R_ERR_INVALID_ARG);
   const bool shared = cfg->I_s > 0;
+  const bool fcomb = fused_combine(cfg);
   C2R_REQUIRE(b->ws && b->ws_bytes >= c2r_workspace_bytes(cfg, C2R_WS_LAYER), C2R_ERR_WORKSPACE);
-  C2R_REQUIRE(b->dY && b->dYp && b->dAB && b->dXp && b->dl && b->dW13p && b->dW2 && b->dWg && b->dX && b->w_row,
+  C2R_REQUIRE(b->dY && b->dYp && b->dAB && (fcomb ? b->dXacc != nullptr : b->dXp != nullptr) && b->dl && b->dW13p &&
+                  b->dW2 && b->dWg && b->dX && b->w_row,
               C2R_ERR_INVALID_ARG);
-  if (shared) C2R_REQUIRE(b->dABs && b->dXs && b->dz && b->dWs13p && b->dWs2 && b->dwsg, C2R_ERR_INVALID_ARG);
+  if (shared) C2R_REQUIRE(b->dABs && (fcomb || b->dXs) && b->dz && b->dWs13p && b->dWs2 && b->dwsg, C2R_ERR_INVALID_ARG);
   const int64_t R = permuted_rows(cfg);
   const LayerWs ws = layer_ws(cfg, b->ws);
   const SideStream ss(b, stream, shared);
   if (shared) {
     // the shared expert reads dY as it is; its gate enters through the row scale
+    c2r_expert_opts o{};
+    o.row_scale = b->z; o.scale_kind = C2R_SCALE_SIGMOID; o.qpart = ws.qspart;
     C2R_TRY(ss.fork());
     C2R_TRY(c2r_grouped_swiglu_bwd(cfg, 1, cfg->I_s, cfg->N, b->X, b->s_counts, b->s_offsets, b->Ws13p, b->Ws2, b->ABs,
-                                   b->Hs, b->dY, b->z, C2R_SCALE_SIGMOID, b->dABs, b->dXs, b->dWs13p, b->dWs2, ws.qspart,
-                                   accumulate, b->status, ss.work()));
+                                   b->Hs, b->dY, b->dABs, fcomb ? (void*)b->dXacc : b->dXs, b->dWs13p, b->dWs2, accumulate,
+                                   &o, b->status, ss.work()));
+  } else if (fcomb) {
+    C2R_CUDA(cudaMemsetAsync(b->dXacc, 0, sizeof(float) * (size_t)cfg->N * cfg->d, as_stream(stream)));
   }
   // transpose of the combine's gather: every permuted row receives its token's dY unchanged
   C2R_TRY(c2r_permute_rows(cfg, b->dY, b->row_of_slot, b->counts, b->offsets, b->dYp, stream));
-  if (gather_fused(cfg, b->X))
-    C2R_TRY(c2r_grouped_swiglu_bwd_gather(cfg, cfg->E, cfg->I, R, b->X, b->slot_of_row, b->counts, b->offsets, b->W13p,
-                                          b->W2, b->AB, b->H, b->dYp, b->w_row, C2R_SCALE_ROW, b->dAB, b->dXp, b->dW13p,
-                                          b->dW2, ws.qpart, accumulate, b->status, stream));
-  else
-    C2R_TRY(c2r_grouped_swiglu_bwd(cfg, cfg->E, cfg->I, R, b->Xp, b->counts, b->offsets, b->W13p, b->W2, b->AB, b->H,
-                                   b->dYp, b->w_row, C2R_SCALE_ROW, b->dAB, b->dXp, b->dW13p, b->dW2, ws.qpart, accumulate,
-                                   b->status, stream));
-  C2R_TRY(ss.join());
+  const bool gfused = gather_fused(cfg, b->X);
+  c2r_expert_opts o{};
+  o.row_scale = b->w_row; o.scale_kind = C2R_SCALE_ROW; o.qpart = ws.qpart;
+  if (gfused) { o.X = b->X; o.slot_of_row = b->slot_of_row; }
+  if (fcomb) {
+    o.token_acc = b->dXacc; o.slot_of_row = b->slot_of_row;
+    C2R_TRY(ss.join());  // the shared expert's dX term is in the accumulator before the routed rows are added
+  }
+  C2R_TRY(c2r_grouped_swiglu_bwd(cfg, cfg->E, cfg->I, R, gfused ? nullptr : b->Xp, b->counts, b->offsets, b->W13p, b->W2,
+                                 b->AB, b->H, b->dYp, b->dAB, fcomb ? nullptr : b->dXp, b->dW13p, b->dW2, accumulate, &o,
+                                 b->status, stream));
+  if (!fcomb) C2R_TRY(ss.join());
   C2R_TRY(c2r_route_bwd_scaled(cfg, b->w, b->row_of_slot, ws.qpart, ws.nq, shared ? b->z : nullptr, ws.qspart, ws.nqs, b->dw,
                                b->dl, shared ? b->dz : nullptr, stream));
   C2R_TRY(c2r_gate_bwd(cfg, b->X, b->Xp, b->counts, b->offsets, b->slot_of_row, b->dl, shared ? b->dz : nullptr,
                        b->dWg, shared ? b->dwsg : nullptr, accumulate, ws.gate_bwd, align256(gate_bwd_ws_bytes(cfg)),
                        stream));
-  C2R_TRY(c2r_unpermute_grad(cfg, b->dXp, b->row_of_slot, shared ? b->dXs : nullptr, b->idx, b->dl, b->Wg,
+  C2R_TRY(c2r_unpermute_grad(cfg, fcomb ? nullptr : b->dXp, b->row_of_slot,
+                             fcomb ? (void*)b->dXacc : (shared ? b->dXs : nullptr), b->idx, b->dl, b->Wg,
                              shared ? b->dz : nullptr, shared ? b->wsg : nullptr, b->dX, 0, stream));
   return C2R_OK;
 }

@@ -27,6 +27,9 @@ struct SimtGemm {
   int scale_kind;
   float* qpart;            // SIMT_EPI_SWIGLU_BWD: [ceil(I / 64)][R] partial row dots, or NULL
   long long R;
+  float* token_acc;        // SIMT_EPI_STORE: add row r into token_acc[slot_of_row[r] / slots_per_token] instead of storing
+  const int32_t* slot_of_row;
+  int slots_per_token;
   const int32_t* counts;
   const int32_t* offsets;
   long long sam, sak, sbn, sbk, sB, sC, ldc;
@@ -57,9 +60,11 @@ struct SwigluCall {
   float* qpart;  // backward: [swiglu_qparts][R] partial row dots <dH_r, H_r>, or NULL
   int accumulate;
   int32_t* status;
-  // gather-fused dispatch (both or neither): rows of the permuted operand are fetched from X inside the kernels
+  // gather-fused dispatch (X with slot_of_row): rows of the permuted operand are fetched from X inside the kernels
   const void* X;
   const int32_t* slot_of_row;
+  // fused combine (token_acc with slot_of_row): the [R,d] float result is added into token_acc[slot_of_row[r] / K]
+  float* token_acc;
 };
 
 template <typename T>

@@ -134,7 +134,11 @@ __global__ void __launch_bounds__(256) simt_gemm_kernel(SimtGemm g) {
       const int n = n0 + tx * 4 + j;
       if (n >= g.Ndim) continue;
       float v = acc[i][j];
-      if (g.epi == SIMT_EPI_STORE) {
+      if (g.epi == SIMT_EPI_STORE && g.token_acc != nullptr) {
+        // fused combine: the row is added into its token's accumulator (fp32 atomics, order not fixed)
+        const int sl = g.slot_of_row[r0 + m];
+        if (sl >= 0) atomicAdd(g.token_acc + (long long)(sl / g.slots_per_token) * g.ldc + n, v);
+      } else if (g.epi == SIMT_EPI_STORE) {
         TC* o = C + (long long)m * g.ldc + n;
         if (g.accumulate) v += to_f32(*o);
         *o = from_f32<TC>(v);
@@ -199,6 +203,7 @@ int simt_swiglu_fwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) 
   // Yp = H W2^T  (fp32 partial result)
   g.A = a.H; g.sam = I; g.sak = 1; g.B = a.W2; g.sbn = I; g.sbk = 1; g.sB = (long long)d * I;
   g.C = a.Yp; g.ldc = d; g.Ndim = d; g.Kdim = I;
+  g.token_acc = a.token_acc; g.slot_of_row = a.slot_of_row; g.slots_per_token = cfg->K;
   return simt_launch<T, float>(g, a.nE, max_m, s);
 }
 
@@ -219,8 +224,10 @@ int simt_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) 
   g.epi = SIMT_EPI_STORE; g.aux = nullptr; g.aux2 = nullptr; g.qpart = nullptr; g.row_scale = nullptr; g.scale_kind = 0;
   g.A = a.dAB; g.sam = 2 * I; g.sak = 1; g.B = a.W13p; g.sbn = 1; g.sbk = d; g.sB = (long long)2 * I * d;
   g.C = a.dXp; g.ldc = d; g.Ndim = d; g.Kdim = 2 * I;
+  g.token_acc = a.token_acc; g.slot_of_row = a.slot_of_row; g.slots_per_token = cfg->K;
   rc = simt_launch<T, float>(g, nE, max_m, s);
   if (rc) return rc;
+  g.token_acc = nullptr;
   // dW2_e = dYp_e^T H_e   [d, I]
   g.mode = SIMT_WGRAD; g.accumulate = a.accumulate;
   g.A = a.dYp; g.sam = 1; g.sak = d; g.B = a.H; g.sbn = 1; g.sbk = I;

@@ -56,6 +56,7 @@ struct TcParams {
   const float* row_scale;
   int scale_kind;
   float* qpart;    // TC_EPI_SWIGLU_BWD: [2 * n_tiles][R] partial row dots <dH_r, H_r>, or NULL
+  float* token_acc;  // TC_EPI_F32: add row r into token_acc[slot_of_row[r] / slots_per_token, :] instead of storing it
   // row-gathering variants: the operand's rows are token rows of X picked through slot_of_row
   const int32_t* slot_of_row;  // [R], -1 = padding (reads zeros)
   int slots_per_token;         // K of the routing
@@ -170,6 +171,42 @@ __device__ __forceinline__ void stage_to_global(uint32_t buf, uint8_t* g, long l
     if (row < rows_valid) *reinterpret_cast<uint4*>(g + row * pitch + 16 * chunk) = lds128(stg_addr(buf, row, chunk));
   }
 }
+// Staging tile (fp32) -> added into rows of an fp32 array starting at g (row pitch in bytes): the row of the tile
+// held by lane l goes to row tok_mine of lane l; a negative token skips the row.  Vector reductions of 16 bytes,
+// 4 rows x 128 bytes per instruction.  Every lane of the warp must call.
+__device__ __forceinline__ void stage_red_to_rows(uint32_t buf, uint8_t* g, long long pitch, int tok_mine, int valid_bytes,
+                                                  int lane) {
+  const int chunk = lane & 7, sub = lane >> 3;
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int row = 4 * it + sub;
+    const int tok = __shfl_sync(0xffffffffu, tok_mine, row);
+    if (tok >= 0 && 16 * chunk < valid_bytes) {
+      const uint4 v = lds128(stg_addr(buf, row, chunk));
+      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(g + (long long)tok * pitch + 16 * chunk),
+                   "f"(__uint_as_float(v.x)), "f"(__uint_as_float(v.y)), "f"(__uint_as_float(v.z)), "f"(__uint_as_float(v.w))
+                   : "memory");
+    }
+  }
+}
+// Global rows [0, rows_valid) x bytes [0, valid_bytes) -> staging tile, asynchronously (16-byte cp.async per lane and
+// row, no registers involved); zeros elsewhere.  Complete after async_copies_wait() + __syncwarp().
+__device__ __forceinline__ void global_rows_to_stage_async(uint32_t buf, const uint8_t* g, long long pitch, int rows_valid,
+                                                           int valid_bytes, int lane) {
+  const int chunk = lane & 7, sub = lane >> 3;
+#pragma unroll
+  for (int it = 0; it < 8; ++it) {
+    const int row = 4 * it + sub;
+    const bool live = row < rows_valid && 16 * chunk < valid_bytes;
+    const uint8_t* src = live ? g + row * pitch + 16 * chunk : g;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(stg_addr(buf, row, chunk)), "l"(src),
+                 "r"(live ? 16 : 0)
+                 : "memory");
+  }
+}
+__device__ __forceinline__ void async_copies_wait() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
 // Global rows [0, rows_valid) x bytes [0, valid_bytes) -> registers in the row-contiguous shape
 // (v[it] = chunk (lane & 7) of row 4*it + (lane >> 3)); zeros elsewhere.
 __device__ __forceinline__ void global_rows_load(uint4 (&v)[8], const uint8_t* g, long long pitch, int rows_valid,
@@ -210,7 +247,8 @@ __device__ __forceinline__ float row_scale_of(const TcParams& p, long long r, bo
 // GATHER: 0 = both operands are plain arrays; 1 = A's rows (TC_ROWS, K-major) are token rows gathered from X;
 // 2 = B's contraction rows (TC_WGRAD, MN-major) are token rows gathered from X.  map_a / map_b is then the
 // one-row-box map of X, and the permuted copy of X is never needed.
-template <bool A_MN, bool B_MN, int GATHER>
+// EPI: the epilogue (TC_EPI_*), a template parameter so that every form gets its own register allocation.
+template <bool A_MN, bool B_MN, int GATHER, int EPI>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -425,7 +463,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const long long mrow = row0 + lane;
       bool waited = !have_acc;
       const float sc = row_scale_of(p, mrow, lane < rows_valid);  // requested before the accumulator is awaited
-      if (p.epi == TC_EPI_SWIGLU_BWD) {
+      int tok_mine = -1;  // fused combine: the token this lane's row belongs to
+      if (EPI == TC_EPI_F32 && p.token_acc != nullptr && lane < rows_valid) {
+        const int sl = p.slot_of_row[mrow];
+        tok_mine = sl >= 0 ? sl / p.slots_per_token : -1;
+      }
+      if constexpr (EPI == TC_EPI_SWIGLU_BWD) {
         // dA = s_r dH (dH/dA), dB = s_r dH (dH/dB) on groups of 64 H columns, s_r the row's scale; the forward pass
         // saved both local derivatives.  With qpart, also the row dot <dH_r, H_r> over this warp's columns (H as the
         // forward stored it, scale included): the gradient w.r.t. the scale times the scale.  None of the loads
@@ -442,41 +485,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const long long pitch = 4ll * p.I;  // bytes per row of AB / dAB
           const uint8_t* gsrc = (const uint8_t*)p.AB + row0 * pitch;
           uint8_t* go = (uint8_t*)p.C + row0 * pitch;
-          // Loads are requested ahead of their use, but staged one piece at a time so that at most two pieces
-          // (64 registers) are in flight per thread.
-          uint4 in0[8], in1[8];
-          if (want_q) {  // the H piece, for the row dots
-            global_rows_load(in1, (const uint8_t*)p.H + row0 * (2ll * p.I) + 2 * hc0, 2ll * p.I, rows_valid, vbytes, lane);
-            stage_rows_store(buf1, in1, lane);
+          // The two saved derivatives travel global -> staging tile asynchronously; the H piece (row dots) is read
+          // straight into registers, every lane its own row.  All of it is in flight at once.
+          global_rows_to_stage_async(buf0, gsrc + 2 * col_a, pitch, rows_valid, vbytes, lane);
+          global_rows_to_stage_async(buf1, gsrc + 2 * col_b, pitch, rows_valid, vbytes, lane);
+          uint4 hrow[8];
+          if (want_q) {
+            const uint8_t* hp = (const uint8_t*)p.H + mrow * (2ll * p.I) + 2 * hc0;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+              hrow[c] = (lane < rows_valid && 16 * c < vbytes) ? *reinterpret_cast<const uint4*>(hp + 16 * c) : make_uint4(0, 0, 0, 0);
           }
-          global_rows_load(in0, gsrc + 2 * col_a, pitch, rows_valid, vbytes, lane);
-          global_rows_load(in1, gsrc + 2 * col_b, pitch, rows_valid, vbytes, lane);
-          stage_rows_store(buf0, in0, lane);
+          async_copies_wait();
           __syncwarp();
           if (!waited) {
             if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
             tc_fence_after();
             waited = true;
           }
-          if (want_q) {
-            // pass 1 over the accumulator columns of the group: q += <dH_r, H_r>
-#pragma unroll
-            for (int pc = 0; pc < 4; ++pc) {
-              if (32 * pc >= vbytes) break;  // warp-uniform
-              uint32_t r0[16];
-              float hv[16];
-              if (have_acc) {
-                tc_ld16(taddr_row + 64 * g + 16 * pc, r0);
-                tc_ld_wait();
-              }
-              unpack_bf16x16(lds128(stg_addr(buf1, lane, 2 * pc)), lds128(stg_addr(buf1, lane, 2 * pc + 1)), hv);
-#pragma unroll
-              for (int i = 0; i < 16; ++i) qacc = fmaf(have_acc ? __uint_as_float(r0[i]) : 0.f, hv[i], qacc);
-            }
-            __syncwarp();
-          }
-          stage_rows_store(buf1, in1, lane);
-          __syncwarp();
 #pragma unroll
           for (int pc = 0; pc < 4; ++pc) {
             if (32 * pc >= vbytes) break;  // warp-uniform
@@ -487,13 +513,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               tc_ld_wait();
             }
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v0[i] = have_acc ? sc * __uint_as_float(r0[i]) : 0.f;
+            for (int i = 0; i < 16; ++i) v0[i] = have_acc ? __uint_as_float(r0[i]) : 0.f;
+            if (want_q) {
+              float hv[16];
+              unpack_bf16x16(hrow[2 * pc], hrow[2 * pc + 1], hv);
+#pragma unroll
+              for (int i = 0; i < 16; ++i) qacc = fmaf(v0[i], hv[i], qacc);
+            }
             const uint32_t sa0 = stg_addr(buf0, lane, 2 * pc), sa1 = stg_addr(buf0, lane, 2 * pc + 1);
             const uint32_t sb0 = stg_addr(buf1, lane, 2 * pc), sb1 = stg_addr(buf1, lane, 2 * pc + 1);
             unpack_bf16x16(lds128(sa0), lds128(sa1), ga);
             unpack_bf16x16(lds128(sb0), lds128(sb1), gb);
 #pragma unroll
-            for (int i = 0; i < 16; ++i) { da[i] = v0[i] * ga[i]; db[i] = v0[i] * gb[i]; }
+            for (int i = 0; i < 16; ++i) { const float v = sc * v0[i]; da[i] = v * ga[i]; db[i] = v * gb[i]; }
             sts128(sa0, pack_bf16x8(da)); sts128(sa1, pack_bf16x8(da + 8));
             sts128(sb0, pack_bf16x8(db)); sts128(sb1, pack_bf16x8(db + 8));
           }
@@ -510,7 +542,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (!mbar_wait(tfull0 + 8 * acc, acc_phase, abort_flag)) { ok = false; break; }
         tc_fence_after();
       }
-      if (p.epi == TC_EPI_SWIGLU_FWD) {
+      if constexpr (EPI == TC_EPI_SWIGLU_FWD) {
         // accumulator columns [0,w) = gate (A), [w,2w) = up (B): H = silu(A) * B, and for the backward pass
         // its local derivatives dH/dA = B silu'(A) (gate columns of the packed buffer) and dH/dB = silu(A) (up columns)
         const int n_groups = (w + 63) >> 6;
@@ -561,7 +593,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             __syncwarp();
           }
         }
-      } else if (p.epi == TC_EPI_F32) {
+      } else if constexpr (EPI == TC_EPI_F32) {
         const int n_groups = (w + 31) >> 5;  // 32 fp32 columns = 128 bytes
         for (int g = hsel; g < n_groups; g += 2) {
           const int c = 32 * g;
@@ -581,11 +613,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                      have_acc ? make_uint4(r0[4 * i], r0[4 * i + 1], r0[4 * i + 2], r0[4 * i + 3]) : make_uint4(0, 0, 0, 0));
           }
           __syncwarp();
-          stage_to_global(buf, (uint8_t*)p.C + row0 * (4 * p.ldc) + 4ll * (TILE_N * ti.jn + c), 4 * p.ldc, rows_valid, vbytes,
-                          lane);
+          if (p.token_acc != nullptr)
+            stage_red_to_rows(buf, (uint8_t*)p.token_acc + 4ll * (TILE_N * ti.jn + c), 4 * p.ldc, tok_mine, vbytes, lane);
+          else
+            stage_to_global(buf, (uint8_t*)p.C + row0 * (4 * p.ldc) + 4ll * (TILE_N * ti.jn + c), 4 * p.ldc, rows_valid, vbytes,
+                            lane);
         }
         __syncwarp();
-      } else if (p.epi == TC_EPI_WGRAD_BF16) {
+      } else if constexpr (EPI == TC_EPI_WGRAD_BF16) {
         const int n_groups = (w + 63) >> 6;
         for (int g = hsel; g < n_groups; g += 2) {
           const int c = 64 * g;
@@ -624,7 +659,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           }
         }
         __syncwarp();
-      } else if (p.epi == TC_EPI_T_F32) {
+      } else if constexpr (EPI == TC_EPI_T_F32) {
         // transposed fp32 store out[group][column][row]: a warp's 32 rows are contiguous in memory
         float* obase = (float*)p.C + (long long)ti.expert * p.sC + mrow;
         for (int ci = hsel; ci < (w >> 4); ci += 2) {
@@ -663,7 +698,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-template <bool A_MN, bool B_MN, int GATHER = 0>
+template <bool A_MN, bool B_MN, int EPI, int GATHER = 0>
 static int launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& p, cudaStream_t s) {
   constexpr int smem = SMEM_BYTES;
   constexpr int MAX_DEV = 64;
@@ -684,17 +719,17 @@ static int launch(const CUtensorMap& ma, const CUtensorMap& mb, const TcParams& 
   cfg.numAttrs = 1;
   int grid = __atomic_load_n(&grid_of_device[dev], __ATOMIC_ACQUIRE);
   if (grid == 0) {
-    C2R_CUDA(cudaFuncSetAttribute(tc_gemm_kernel<A_MN, B_MN, GATHER>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    C2R_CUDA(cudaFuncSetAttribute(tc_gemm_kernel<A_MN, B_MN, GATHER, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     int sms = 0, pairs = 0;
     C2R_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     cfg.gridDim = dim3(sms / 2 * 2);
-    C2R_CUDA(cudaOccupancyMaxActiveClusters(&pairs, tc_gemm_kernel<A_MN, B_MN, GATHER>, &cfg));
+    C2R_CUDA(cudaOccupancyMaxActiveClusters(&pairs, tc_gemm_kernel<A_MN, B_MN, GATHER, EPI>, &cfg));
     if (pairs < 1) return C2R_ERR_UNSUPPORTED_SHAPE;
     grid = 2 * (pairs < sms / 2 ? pairs : sms / 2);
     __atomic_store_n(&grid_of_device[dev], grid, __ATOMIC_RELEASE);
   }
   cfg.gridDim = dim3(grid);
-  C2R_CUDA(cudaLaunchKernelEx(&cfg, tc_gemm_kernel<A_MN, B_MN, GATHER>, ma, mb, p));
+  C2R_CUDA(cudaLaunchKernelEx(&cfg, tc_gemm_kernel<A_MN, B_MN, GATHER, EPI>, ma, mb, p));
   C2R_LAUNCH_CHECK();
   return C2R_OK;
 }
@@ -725,7 +760,7 @@ int tc_swiglu_fwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
   p.epi = TC_EPI_SWIGLU_FWD; p.K = d; p.Nout = I; p.n_tiles = (I + 127) / 128; p.C = a.AB; p.H = a.H;
   p.row_scale = a.row_scale; p.scale_kind = a.row_scale ? a.scale_kind : 0;
   p.slot_of_row = a.slot_of_row; p.slots_per_token = cfg->K; p.n_tokens = cfg->N;
-  rc = gather ? launch<false, false, 1>(ma, mb, p, s) : launch<false, false>(ma, mb, p, s);
+  rc = gather ? launch<false, false, TC_EPI_SWIGLU_FWD, 1>(ma, mb, p, s) : launch<false, false, TC_EPI_SWIGLU_FWD>(ma, mb, p, s);
   if (rc) return rc;
   // Yp = H W2^T (fp32)
   rc = make_map(&ma, a.H, I, R, 0, BK, BM);
@@ -734,7 +769,8 @@ int tc_swiglu_fwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
   if (rc) return rc;
   p.epi = TC_EPI_F32; p.K = I; p.Nout = d; p.n_tiles = (d + TILE_N - 1) / TILE_N; p.C = a.Yp; p.ldc = d; p.H = nullptr;
   p.row_scale = nullptr; p.scale_kind = 0;
-  return launch<false, false>(ma, mb, p, s);
+  p.token_acc = a.token_acc; p.slot_of_row = a.slot_of_row;  // fused combine: rows are added into their tokens
+  return launch<false, false, TC_EPI_F32>(ma, mb, p, s);
 }
 
 int tc_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
@@ -751,7 +787,7 @@ int tc_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
   if (rc) return rc;
   p.epi = TC_EPI_SWIGLU_BWD; p.K = d; p.Nout = I; p.n_tiles = (I + TILE_N - 1) / TILE_N; p.C = a.dAB; p.AB = a.AB;
   p.row_scale = a.row_scale; p.scale_kind = a.row_scale ? a.scale_kind : 0; p.qpart = a.qpart; p.H = a.H;
-  rc = launch<false, true>(ma, mb, p, s);
+  rc = launch<false, true, TC_EPI_SWIGLU_BWD>(ma, mb, p, s);
   if (rc) return rc;
   p.row_scale = nullptr; p.scale_kind = 0; p.qpart = nullptr; p.H = nullptr;
   // dXp = dAB W13p (fp32)
@@ -760,8 +796,10 @@ int tc_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
   rc = make_map(&mb, a.W13p, d, 2 * I, nE, 64, 64);  // W13p_e is [2I (k)][d (n)]: MN-major B
   if (rc) return rc;
   p.epi = TC_EPI_F32; p.K = 2 * I; p.Nout = d; p.n_tiles = (d + TILE_N - 1) / TILE_N; p.C = a.dXp; p.ldc = d; p.AB = nullptr;
-  rc = launch<false, true>(ma, mb, p, s);
+  p.token_acc = a.token_acc; p.slot_of_row = a.slot_of_row; p.slots_per_token = cfg->K;
+  rc = launch<false, true, TC_EPI_F32>(ma, mb, p, s);
   if (rc) return rc;
+  p.token_acc = nullptr;
   // dW2_e = dYp_e^T H_e  [d, I]
   p.mode = TC_WGRAD; p.epi = TC_EPI_WGRAD_BF16; p.accumulate = a.accumulate;
   rc = make_map(&ma, a.dYp, d, R, 0, 64, 64);
@@ -770,7 +808,7 @@ int tc_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
   if (rc) return rc;
   p.Mout = d; p.Nout = I; p.m_tiles = (d + TILE_M - 1) / TILE_M; p.n_tiles = (I + TILE_N - 1) / TILE_N;
   p.C = a.dW2; p.ldc = I; p.sC = (long long)d * I;
-  rc = launch<true, true>(ma, mb, p, s);
+  rc = launch<true, true, TC_EPI_WGRAD_BF16>(ma, mb, p, s);
   if (rc) return rc;
   // dW13p_e = dAB_e^T Xp_e  [2I, d]
   rc = make_map(&ma, a.dAB, 2 * I, R, 0, 64, 64);
@@ -781,7 +819,7 @@ int tc_swiglu_bwd(const c2r_config* cfg, const SwigluCall& a, cudaStream_t s) {
   p.Mout = 2 * I; p.Nout = d; p.m_tiles = (2 * I + TILE_M - 1) / TILE_M; p.n_tiles = (d + TILE_N - 1) / TILE_N;
   p.C = a.dW13p; p.ldc = d; p.sC = (long long)2 * I * d;
   p.slot_of_row = a.slot_of_row; p.slots_per_token = cfg->K; p.n_tokens = cfg->N;
-  return gather ? launch<true, true, 2>(ma, mb, p, s) : launch<true, true>(ma, mb, p, s);
+  return gather ? launch<true, true, TC_EPI_WGRAD_BF16, 2>(ma, mb, p, s) : launch<true, true, TC_EPI_WGRAD_BF16>(ma, mb, p, s);
 }
 
 int tc_gate_wgrad(const c2r_config* cfg, const void* X, const void* dLd, float* partial, int n_splits,
@@ -798,7 +836,7 @@ int tc_gate_wgrad(const c2r_config* cfg, const void* X, const void* dLd, float* 
   if (rc) return rc;
   p.Mout = d; p.Nout = 64; p.m_tiles = (d + TILE_M - 1) / TILE_M; p.n_tiles = 1;
   p.C = partial; p.ldc = d; p.sC = 64ll * d;
-  return launch<true, true>(ma, mb, p, s);
+  return launch<true, true, TC_EPI_T_F32>(ma, mb, p, s);
 }
 
 }  // namespace c2r

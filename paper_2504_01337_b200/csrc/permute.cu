@@ -338,7 +338,7 @@ __device__ __forceinline__ void load_as_float(const S* p, float* f) {
 //          + ecoef(t) * extra[t,:]                           (ecoef = sigmoid(z[t]) if z else 1)
 //          + sum_k dl[t,k] * Wg[idx[t,k],:] + dz[t] * wsg[:] (gate terms, optional)
 //          + out[t,:] if accumulate.
-// src / extra are the fp32 partial results of the expert GEMMs; out has the storage type.
+// src == NULL: no such term (the producer already added its rows into extra).  src / extra are the fp32 partial results of the expert GEMMs; out has the storage type.
 // One warp per token, fp32 accumulation in k order.  Serves the combine and the gradient un-permute.
 template <typename T>
 __global__ void __launch_bounds__(256) gather_sum_kernel(const float* __restrict__ src, const int32_t* __restrict__ rows_g,
@@ -375,13 +375,15 @@ __global__ void __launch_bounds__(256) gather_sum_kernel(const float* __restrict
     float acc[V::N];
 #pragma unroll
     for (int j = 0; j < V::N; ++j) acc[j] = 0.f;
+    if (src != nullptr) {
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      if (k >= K) break;
-      float f[V::N];
-      load_as_float<T, float>(src + (size_t)rows[k] * d + col, f);
+      for (int k = 0; k < 8; ++k) {
+        if (k >= K) break;
+        float f[V::N];
+        load_as_float<T, float>(src + (size_t)rows[k] * d + col, f);
 #pragma unroll
-      for (int j = 0; j < V::N; ++j) acc[j] = fmaf(cf[k], f[j], acc[j]);
+        for (int j = 0; j < V::N; ++j) acc[j] = fmaf(cf[k], f[j], acc[j]);
+      }
     }
     if (extra) {
       float f[V::N];
@@ -759,7 +761,7 @@ extern "C" int c2r_combine(const c2r_config* cfg, const void* Yp, const float* w
                            const void* Ys, const float* z, void* Y, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
-  C2R_REQUIRE(Yp && row_of_slot && Y, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE((Yp || Ys) && row_of_slot && Y, C2R_ERR_INVALID_ARG);
   if (cfg->dtype == C2R_BF16)
     return gather_sum_launch<__nv_bfloat16>(cfg, Yp, row_of_slot, w, Ys, z, nullptr, nullptr, nullptr, nullptr,
                                             nullptr, Y, 0, as_stream(stream));
@@ -772,7 +774,7 @@ extern "C" int c2r_unpermute_grad(const c2r_config* cfg, const void* dXp, const 
                                   const void* wsg, void* dX, int accumulate, void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
-  C2R_REQUIRE(dXp && row_of_slot && dX, C2R_ERR_INVALID_ARG);
+  C2R_REQUIRE((dXp || dXs) && row_of_slot && dX, C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(!dl || (idx && Wg), C2R_ERR_INVALID_ARG);
   C2R_REQUIRE((dz == nullptr) == (wsg == nullptr), C2R_ERR_INVALID_ARG);
   if (cfg->dtype == C2R_BF16)

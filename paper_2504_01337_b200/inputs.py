@@ -118,6 +118,9 @@ WORKLOADS = {
     "c4": Workload("c4", N=16384, d=2048, E=60, I=1408, K=4, T=16, P=4, I_s=5632, n_calib=16384, backward=False, skew=True),
     # c3 shapes on a quarter of the tokens: the small case for profiler captures
     "c3s": Workload("c3s", N=4096, d=2048, E=60, I=1408, K=4, T=16, P=4, I_s=5632, n_calib=4096),
+    # c3's per-expert shape (about 1092 rows per expert) on a quarter of the tokens and experts: < 1 GB on the
+    # device, for profiler captures of the routed GEMM launches
+    "c3e": Workload("c3e", N=4096, d=2048, E=15, I=1408, K=4, T=6, P=3, I_s=5632, n_calib=4096),
     "c5": Workload("c5", N=65536, d=2048, E=60, I=1408, K=4, T=16, P=4, I_s=5632, n_calib=65536),
 }
 

@@ -21,11 +21,11 @@ class C2RLayer:
     to torch tensors."""
 
     def __init__(self, N, d, E, I, K, T, P, I_s=0, bf16=True, row_align=None, backward=True, profile=False,
-                 renorm=1, device="cuda", gather_fused=False, side_stream=False):
+                 renorm=1, device="cuda", gather_fused=False, side_stream=False, fused_combine=False):
         if row_align is None:
             row_align = 128 if bf16 else 1
         self.cfg = B.make_config(N, d, E, I, K, T, P, I_s, B.BF16 if bf16 else B.F32, row_align, renorm,
-                                 B.FLAG_GATHER_FUSED if gather_fused else 0)
+                                 (B.FLAG_GATHER_FUSED if gather_fused else 0) | (B.FLAG_FUSED_COMBINE if fused_combine else 0))
         self.bf16 = bf16
         self.device = device
         self.R = B.permuted_rows(self.cfg)
@@ -49,7 +49,10 @@ class C2RLayer:
         if not (gather_fused and bf16):  # the gather-fused GEMMs read token rows from X: no permuted copy
             t["Xp"] = buf((R, d))
         t["H"] = buf((R, I))
-        t["Yp"] = buf((R, d), f32)
+        if fused_combine:  # the GEMM epilogues add their rows into per-token fp32 accumulators: no Yp / Ys / dXp / dXs
+            t["Yacc"] = buf((N, d), f32)
+        else:
+            t["Yp"] = buf((R, d), f32)
         t["Y"] = buf((N, d))
         t["volume"] = torch.zeros((4 + 2 * P * P,), dtype=torch.int64, device=dev)
         t["status"] = torch.zeros((1,), dtype=i32, device=dev)
@@ -57,7 +60,8 @@ class C2RLayer:
         if I_s:
             t["z"] = buf((N,), f32)
             t["Hs"] = buf((N, I_s))
-            t["Ys"] = buf((N, d), f32)
+            if not fused_combine:
+                t["Ys"] = buf((N, d), f32)
             t["s_counts"] = torch.tensor([N], dtype=i32, device=dev)
             t["s_offsets"] = torch.tensor([0, N], dtype=i32, device=dev)
         if backward:
@@ -67,7 +71,10 @@ class C2RLayer:
             t["dY"] = buf((N, d))
             t["dYp"] = buf((R, d))
             t["dAB"] = buf((R, 2 * I))
-            t["dXp"] = buf((R, d), f32)
+            if fused_combine:
+                t["dXacc"] = buf((N, d), f32)
+            else:
+                t["dXp"] = buf((R, d), f32)
             t["dw"] = buf((N, K), f32)
             t["dl"] = buf((N, K), f32)
             t["dW13p"] = buf((E, 2 * I, d))
@@ -76,7 +83,8 @@ class C2RLayer:
             t["dX"] = buf((N, d))
             if I_s:
                 t["dABs"] = buf((N, 2 * I_s))
-                t["dXs"] = buf((N, d), f32)
+                if not fused_combine:
+                    t["dXs"] = buf((N, d), f32)
                 t["dz"] = buf((N,), f32)
                 t["dWs13p"] = buf((1, 2 * I_s, d))
                 t["dWs2"] = buf((1, d, I_s))

@@ -397,3 +397,39 @@ def test_two_micro_batches_accumulate_every_parameter_gradient():
     for got, k in ((grads[0], "dW1"), (grads[1], "dW3"), (lay.host("dW2"), "dW2"), (lay.host("dWg"), "dWg"),
                    (grads[2], "dWs1"), (grads[3], "dWs3"), (lay.host("dWs2")[0], "dWs2"), (lay.host("dwsg"), "dwsg")):
         assert_close_abs(got, total[k], 2e-4, k)
+
+
+@pytest.mark.parametrize("name,N,d,E,I,K,T,P,I_s,bf16", SMALL + [("bf16-c3-shape", 4096, 2048, 15, 1408, 4, 6, 4, 1408, True)])
+def test_fused_combine_matches_oracle(name, N, d, E, I, K, T, P, I_s, bf16):
+    """C2R_FLAG_FUSED_COMBINE: the down-projection and the dXp GEMM add their rows into per-token fp32 accumulators
+    (no Yp / dXp, no gather pass).  The order of a token's fp32 adds is not fixed, so the comparison is by
+    tolerance, against the oracle, on the same bar as the gather path."""
+    wl = G.Workload(name, N=N, d=d, E=E, I=I, K=K, T=T, P=P, I_s=I_s, bf16=bf16, seed=11)
+    close = _close(bf16)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    Wg = Wg if bf16 else Wg * 8
+    sh = G.shared_weights(wl) if I_s else None
+    sets = random_sets(E, T, seed=5)
+    rank = np.random.default_rng(3).permutation(E)
+    lay = _layer(wl, backward=True, fused_combine=True, side_stream=bool(I_s))
+    assert "Yp" not in lay.t and "dXp" not in lay.t and "Ys" not in lay.t
+    lay.set_params(Wg, W1, W3, W2, wsg, sh)
+    lay.set_routing(mask=mask_of(sets, E), expert_rank=rank)
+    lay.set_input(X, dY)
+    for _ in range(2):  # the accumulators are re-initialised by every pass
+        lay.forward()
+        lay.backward()
+    torch.cuda.synchronize()
+    assert int(lay.t["status"].item()) == 0
+    S = np.arange(N) if N <= 2048 else np.sort(np.random.default_rng(2).choice(N, 512, replace=False))
+    f = O.layer_fwd(X[S], Wg, W1, W3, W2, sets, K, expert_rank=rank, row_align=1, shared=sh, wsg=wsg, logits=lay.host("L")[S])
+    assert np.array_equal(lay.host("idx")[S], f["idx"])
+    close(lay.host("Y")[S], f["Y"], "Y (fused combine)")
+    f2 = O.layer_fwd(X[S], Wg, W1, W3, W2, sets, K, expert_rank=rank, row_align=1, shared=sh, wsg=wsg)
+    same = np.all(f2["idx"] == f["idx"], axis=1)
+    assert same.mean() > 0.9
+    g = O.layer_bwd(X[S], Wg, W1, W3, W2, f2, dY[S], shared=sh, wsg=wsg)
+    close(lay.host("dX")[S][same], g["dX"][same], "dX (fused combine)")
+    _close(bf16, stored_bf16=False)(lay.host("dw")[S][same], g["dw"][same], "dw (fused combine)")
