@@ -325,6 +325,33 @@ def dedup_dispatch_timing(lay, reps=5):
     return res
 
 
+def variant_timing(wl, device, X_host, dY_host, steps, skip):
+    """ms per step of the same training step in the driver configurations the main line does not use: the combine
+    fused into the GEMM epilogues (fp32 adds into per-token accumulators, order not fixed) and the shared expert
+    on a second stream.  Same workload, same inputs, a layer of its own per variant."""
+    import torch
+    res = {}
+    for combine, streams in (("gather", 1), ("gather", 2), ("fused", 1), ("fused", 2)):
+        if (combine, streams) == skip or (streams == 2 and not wl.I_s):
+            continue
+        lay = build_layer(wl, device, fused_combine=combine == "fused", side_stream=streams == 2)
+        lay.set_input(X_host.to(device), dY_host.to(device))
+        for _ in range(3):
+            lay.train_step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            lay.train_step()
+        e1.record()
+        torch.cuda.synchronize()
+        res[f"combine={combine},streams={streams}"] = {"ms_per_step": e0.elapsed_time(e1) / steps, "steps": steps,
+                                                       "status_word": int(lay.t["status"].item())}
+        del lay
+        torch.cuda.empty_cache()
+    return res
+
+
 def skew_report(wl4, device):
     """The skewed-routing stress workload (directly drawn logits with a Zipf-like expert bias and a
     block bonus): profile on its calibration logits, then Top-K vs C2R side by side."""
@@ -415,10 +442,19 @@ def run_reference(args, wl):
     }))
 
 
-# DRAM bytes per launch of tc_gemm_kernel (dram__bytes_read.sum + dram__bytes_write.sum averaged over
-# the 12 expert-GEMM launches of a step) from the ncu launch list of this very command, summarised under
-# profiles/.  Keyed by workload; None where no capture of the current kernel exists.
-GEMM_TRAFFIC_BYTES_PER_LAUNCH = {"c3": 1.035e9}
+def gemm_traffic_bytes_per_launch(workload):
+    """DRAM bytes per launch of tc_gemm_kernel (dram__bytes_read.sum + dram__bytes_write.sum averaged over the
+    expert-GEMM launches of a step) from the table of ncu captures kept under profiles/; None where no
+    capture of the current kernel exists."""
+    path = os.path.join(ROOT, "profiles", "gemm_dram_traffic.md")
+    try:
+        for line in open(path):
+            cells = [c.strip() for c in line.strip().strip("|").split("|")]
+            if len(cells) >= 2 and cells[0] == workload:
+                return float(cells[1])
+    except (OSError, ValueError):
+        pass
+    return None
 
 
 def main():
@@ -436,7 +472,7 @@ def main():
     ap.add_argument("--combine", default="gather", choices=["gather", "fused"],
                     help="gather: the GEMMs store fp32 partials and a gather pass sums them (deterministic); fused: the GEMM "
                          "epilogues add their rows into per-token fp32 accumulators (order of the adds not fixed)")
-    ap.add_argument("--streams", type=int, default=2, choices=[1, 2],
+    ap.add_argument("--streams", type=int, default=1, choices=[1, 2],
                     help="2: the shared expert's GEMMs run on a second stream beside the routing chain")
     ap.add_argument("--dispatch", default="permute", choices=["permute", "gather-fused"],
                     help="permute: c2r_permute writes Xp (faster); gather-fused: the expert GEMMs read token rows from X, no permuted copy")
@@ -588,7 +624,7 @@ def main():
             ach = fl_step / (gemm_ms * 1e-3) / 1e12
             peak = peaks["bf16_tflops_sustained"]
             out["roofline"] = {"bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                               "frac": ach / peak, "traffic": GEMM_TRAFFIC_BYTES_PER_LAUNCH.get(wl.name),
+                               "frac": ach / peak, "traffic": gemm_traffic_bytes_per_launch(wl.name),
                                "peak_source": peaks["source"] + " sustained (bf16_tflops_sustained; burst %.0f)" % peaks["bf16_tflops"],
                                "kernel": "tc_gemm_kernel (grouped SwiGLU GEMMs, routed + shared, fwd + bwd)",
                                "launches_per_step": n_launch, "avg_launch_ms": gemm_ms / n_launch,
@@ -608,6 +644,8 @@ def main():
                                                      cal["C"].cpu(), wl.E, wl.K, wl.T)
             out["skew_report_c4"] = skew_report(G.WORKLOADS["c4"], device)
             out["dedup_dispatch"] = dedup_dispatch_timing(lay)
+            out["variants"] = variant_timing(wl, device, X_host, dY_host, steps=max(3, min(args.steps, 20)),
+                                             skip=(args.combine, args.streams))
         if not args.no_cpu_baseline and world == 1:
             n_tok = args.cpu_baseline_tokens
             _, st = cpu_oracle_step(wl, n_tok)      # builds the inputs (and warms the BLAS threads)

@@ -147,6 +147,10 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     if (!ok && lane == 0) { *abort_flag = 1; if (status) atomicOr(status, C2R_STATUS_WAIT_TIMEOUT); }
   }
 
+  // after a wait gave up, let TMA loads still in flight land before the CTA (and its shared memory) goes away
+  __syncthreads();
+  if (*abort_flag)
+    for (int i = 0; i < 128; ++i) __nanosleep(2000);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

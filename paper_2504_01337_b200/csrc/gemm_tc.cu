@@ -685,6 +685,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (!ok && lane == 0) { *abort_flag = 1; if (p.status) atomicOr(p.status, C2R_STATUS_WAIT_TIMEOUT); }
   }
 
+  // After a wait gave up, TMA loads nobody will wait for may still be in flight towards this CTA's shared memory:
+  // give them time to land (they complete within microseconds) before the CTA can exit.  The peer is held at the
+  // cluster barrier meanwhile, so its shared memory outlives its own stragglers too.
+  __syncthreads();
+  if (*abort_flag)
+    for (int i = 0; i < 128; ++i) __nanosleep(2000);
   // Both CTAs are done with each other's shared and tensor memory before either leaves.
   tc_fence_before();
   __syncthreads();
