@@ -72,7 +72,8 @@ def measured_peaks():
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw")
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap,power.draw,"
+         "clocks_event_reasons.active")
 
     def __init__(self, index):
         self.index, self.proc, self.lines = index, None, []
@@ -107,7 +108,7 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         import datetime
-        sm, mx, pw, reasons = [], [], [], set()
+        sm, mx, pw, reasons, masks = [], [], [], set(), set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
             p = [x.strip() for x in ln.split(",")]
@@ -127,8 +128,11 @@ class ClockSampler:
             for n, v in zip(names, p[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
+            if len(p) > 8 and p[8].lower().startswith("0x"):
+                masks.add(p[8].lower())
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons)}
+                "samples": len(sm), "power_w_max": max(pw) if pw else None, "reasons": sorted(reasons),
+                "active_masks": sorted(masks)}
 
 
 def build_layer(wl, device, profile=True, keep=False, gather_fused=False, fused_combine=False, side_stream=False):
@@ -466,6 +470,8 @@ def main():
     ap.add_argument("--impl", default="c2r", choices=["c2r", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=128)
     ap.add_argument("--cpu-baseline-tokens", type=int, default=1024)
+    ap.add_argument("--min-warmup-s", type=float, default=1.0,
+                    help="keep warming up (beyond --warmup steps) until this much wall time has passed")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
     ap.add_argument("--no-reports", action="store_true", help="skip the Top-K vs C2R dispatch reports")
@@ -519,10 +525,19 @@ def main():
     # ---- device-resident timing ----------------------------------------------------------------
     sampler = ClockSampler(local)
     sampler.start()
+    # Warm-up: the W steps asked for, then more of the same step until the device has been busy for about a
+    # second, so that the timed steps run in the sustained (power-capped) state the roofline's denominator was
+    # measured in instead of the first tenths of a second after idle, when clocks are still settling.
     warm = max(args.warmup, 3)
+    t_warm = time.perf_counter()
     for _ in range(warm):
         lay.train_step()
     torch.cuda.synchronize()
+    while time.perf_counter() - t_warm < args.min_warmup_s:
+        for _ in range(10):
+            lay.train_step()
+        warm += 10
+        torch.cuda.synchronize()
     RP.barrier()
     sampler.mark_begin()
     launches0 = int(lib_launches()) if lib_launches else 0
