@@ -329,7 +329,24 @@ def dedup_dispatch_timing(lay, reps=5):
     return res
 
 
-def variant_timing(wl, device, X_host, dY_host, steps, skip):
+def warm_up(lay, steps, min_s):
+    """`steps` training steps, then more until the device has been busy for `min_s` seconds: the timed steps that
+    follow then run in the sustained (power-capped) state, not in the first tenths of a second after idle.
+    Returns the number of steps run."""
+    import torch
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        lay.train_step()
+    torch.cuda.synchronize()
+    while time.perf_counter() - t0 < min_s:
+        for _ in range(10):
+            lay.train_step()
+        steps += 10
+        torch.cuda.synchronize()
+    return steps
+
+
+def variant_timing(wl, device, X_host, dY_host, steps, skip, min_s=1.0):
     """ms per step of the same training step in the driver configurations the main line does not use: the combine
     fused into the GEMM epilogues (fp32 adds into per-token accumulators, order not fixed) and the shared expert
     on a second stream.  Same workload, same inputs, a layer of its own per variant."""
@@ -340,8 +357,7 @@ def variant_timing(wl, device, X_host, dY_host, steps, skip):
             continue
         lay = build_layer(wl, device, fused_combine=combine == "fused", side_stream=streams == 2)
         lay.set_input(X_host.to(device), dY_host.to(device))
-        for _ in range(3):
-            lay.train_step()
+        warm_up(lay, 3, min_s)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record()
@@ -528,16 +544,7 @@ def main():
     # Warm-up: the W steps asked for, then more of the same step until the device has been busy for about a
     # second, so that the timed steps run in the sustained (power-capped) state the roofline's denominator was
     # measured in instead of the first tenths of a second after idle, when clocks are still settling.
-    warm = max(args.warmup, 3)
-    t_warm = time.perf_counter()
-    for _ in range(warm):
-        lay.train_step()
-    torch.cuda.synchronize()
-    while time.perf_counter() - t_warm < args.min_warmup_s:
-        for _ in range(10):
-            lay.train_step()
-        warm += 10
-        torch.cuda.synchronize()
+    warm = warm_up(lay, max(args.warmup, 3), args.min_warmup_s)
     RP.barrier()
     sampler.mark_begin()
     launches0 = int(lib_launches()) if lib_launches else 0
@@ -660,7 +667,7 @@ def main():
             out["skew_report_c4"] = skew_report(G.WORKLOADS["c4"], device)
             out["dedup_dispatch"] = dedup_dispatch_timing(lay)
             out["variants"] = variant_timing(wl, device, X_host, dY_host, steps=max(3, min(args.steps, 20)),
-                                             skip=(args.combine, args.streams))
+                                             skip=(args.combine, args.streams), min_s=args.min_warmup_s)
         if not args.no_cpu_baseline and world == 1:
             n_tok = args.cpu_baseline_tokens
             _, st = cpu_oracle_step(wl, n_tok)      # builds the inputs (and warms the BLAS threads)
