@@ -79,7 +79,7 @@ __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) {
   return (va > vb) || (va == vb && ia < ib);
 }
 
-constexpr int ROUTE_WARPS = 16;
+constexpr int ROUTE_WARPS = 32;
 
 // A block owns tokens_per_block consecutive tokens (the blocking of the dispatch's counting sort), a warp
 // every ROUTE_WARPS-th of them.  block_counts (optional): [blocks][E] experts' slot counts of the block's
@@ -198,30 +198,31 @@ __global__ void route_bwd_kernel(const float* __restrict__ w, const float* __res
 // S = sum_j q_j:  dl_k = w_k (dw_k - sum_j w_j dw_j) = q_k - w_k S  -- no division by a weight that may be 0.
 // dw (optional, informational) = q_k / w_k where w_k > 0.  Shared expert: q_s = g dL/dg, dz = q_s (1 - g).
 // Partials are added in index order.
-__global__ void __launch_bounds__(256) route_bwd_scaled_kernel(const float* __restrict__ w,
-                                                               const int32_t* __restrict__ row_of_slot,
-                                                               const float* __restrict__ qpart, int nq, long long R,
-                                                               const float* __restrict__ z,
-                                                               const float* __restrict__ qspart, int nqs,
-                                                               float* __restrict__ dw, float* __restrict__ dl,
-                                                               float* __restrict__ dz, int N, int K) {
-  const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= N) return;
-  float q[8];
-  float S = 0.f;
-  for (int k = 0; k < K; ++k) {
+constexpr int RBS_TOKENS = 64;  // tokens per block; one thread per slot
+__global__ void __launch_bounds__(RBS_TOKENS * 8) route_bwd_scaled_kernel(const float* __restrict__ w,
+                                                                          const int32_t* __restrict__ row_of_slot,
+                                                                          const float* __restrict__ qpart, int nq,
+                                                                          long long R, const float* __restrict__ z,
+                                                                          const float* __restrict__ qspart, int nqs,
+                                                                          float* __restrict__ dw, float* __restrict__ dl,
+                                                                          float* __restrict__ dz, int N, int K) {
+  __shared__ float s_q[RBS_TOKENS * 8];
+  const int lt = threadIdx.x / K, k = threadIdx.x - lt * K;  // token of the block, slot of the token
+  const int t = blockIdx.x * RBS_TOKENS + lt;
+  float q = 0.f;
+  if (t < N) {
     const long long row = row_of_slot[(size_t)t * K + k];
-    float acc = 0.f;
-    for (int j = 0; j < nq; ++j) acc += qpart[(long long)j * R + row];
-    q[k] = acc;
-    S += acc;
+    for (int j = 0; j < nq; ++j) q += qpart[(long long)j * R + row];
   }
-  for (int k = 0; k < K; ++k) {
-    const float wk = w[(size_t)t * K + k];
-    dl[(size_t)t * K + k] = q[k] - wk * S;
-    if (dw != nullptr) dw[(size_t)t * K + k] = wk > 0.f ? q[k] / wk : 0.f;
-  }
-  if (dz != nullptr) {
+  s_q[threadIdx.x] = q;
+  __syncthreads();
+  if (t >= N) return;
+  float S = 0.f;
+  for (int j = 0; j < K; ++j) S += s_q[lt * K + j];  // slot order
+  const float wk = w[(size_t)t * K + k];
+  dl[(size_t)t * K + k] = q - wk * S;
+  if (dw != nullptr) dw[(size_t)t * K + k] = wk > 0.f ? q / wk : 0.f;
+  if (dz != nullptr && k == 0) {
     float acc = 0.f;
     for (int j = 0; j < nqs; ++j) acc += qspart[(long long)j * N + t];
     const float g = 1.0f / (1.0f + expf(-z[t]));
@@ -419,7 +420,7 @@ extern "C" int c2r_route_bwd_scaled(const c2r_config* cfg, const float* w, const
   C2R_REQUIRE(!dz || (z && qspart && nqs >= 0), C2R_ERR_INVALID_ARG);
   C2R_REQUIRE(cfg->renorm == 1, C2R_ERR_UNSUPPORTED_SHAPE);
   if (cfg->N == 0) return C2R_OK;
-  route_bwd_scaled_kernel<<<(cfg->N + 255) / 256, 256, 0, as_stream(stream)>>>(w, row_of_slot, qpart, nq, permuted_rows(cfg),
+  route_bwd_scaled_kernel<<<(cfg->N + RBS_TOKENS - 1) / RBS_TOKENS, RBS_TOKENS * cfg->K, 0, as_stream(stream)>>>(w, row_of_slot, qpart, nq, permuted_rows(cfg),
                                                                               z, qspart, nqs, dw, dl, dz, cfg->N, cfg->K);
   C2R_LAUNCH_CHECK();
   return C2R_OK;
