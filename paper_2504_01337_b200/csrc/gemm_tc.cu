@@ -73,16 +73,18 @@ struct TileInfo {
 };
 
 // Decode linear tile id `t`.  s_pt[e] = number of pair tiles of the experts before e (TC_ROWS).
-// Returns false when t is past the last tile.
+// Returns false when t is past the last tile.  e_hint: the expert of the tile this role decoded last (a role walks
+// its tiles in increasing order, so the search for the expert resumes there instead of starting at expert 0).
 __device__ __forceinline__ bool decode_tile(const TcParams& p, const int* s_off, const int* s_cnt, const int* s_pt,
-                                            long long t, TileInfo& ti) {
+                                            long long t, TileInfo& ti, int& e_hint) {
   if (p.mode == TC_ROWS) {
     const long long total = (long long)s_pt[p.n_experts] * p.n_tiles;
     if (t >= total) return false;
     const int mp = (int)(t / p.n_tiles);
     ti.jn = (int)(t % p.n_tiles);
-    int e = 0;
+    int e = (e_hint < p.n_experts && s_pt[e_hint] <= mp) ? e_hint : 0;
     while (e + 1 < p.n_experts && s_pt[e + 1] <= mp) ++e;
+    e_hint = e;
     ti.expert = e;
     ti.m0 = s_off[e] + TILE_M * (mp - s_pt[e]);
     ti.m_end = min(p.R, s_off[e] + (s_cnt[e] + BM - 1) / BM * BM);
@@ -306,9 +308,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t full_mma0 = map_to_cta(full0, 0);  // completion bytes are counted where the MMAs are issued
         uint32_t stage = 0, phase = 0;
         bool ok = true;
+        int e_hint = 0;
         for (long long t = pair_id; ok; t += n_pairs) {
           TileInfo ti;
-          if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti)) break;
+          if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti, e_hint)) break;
           int n_mma, w, brow0;
           n_geometry(p, ti.jn, n_mma, w, brow0);
           const int a0 = ti.m0 + BM * (int)rank;               // this CTA's A rows (or output-row range for MN-major A)
@@ -348,9 +351,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t full_mma0 = map_to_cta(full0, 0);  // completion bytes are counted where the MMAs are issued
         uint32_t stage = 0, phase = 0;
         bool ok = true;
+        int e_hint = 0;
         for (long long t = pair_id; ok; t += n_pairs) {
           TileInfo ti;
-          if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti)) break;
+          if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti, e_hint)) break;
           int n_mma, w, brow0;
           n_geometry(p, ti.jn, n_mma, w, brow0);
           const int a0 = ti.m0 + BM * (int)rank;               // this CTA's A rows (or output-row range for MN-major A)
@@ -408,9 +412,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t stage = 0, phase = 0;
       uint32_t acc = 0, acc_phase = 0;
       bool ok = true;
-      for (long long t = pair_id; ok; t += n_pairs) {
+      int e_hint = 0;
+        for (long long t = pair_id; ok; t += n_pairs) {
         TileInfo ti;
-        if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti)) break;
+        if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti, e_hint)) break;
         if (ti.kblocks == 0) continue;  // empty contraction: the epilogue writes zeros on its own
         int n_mma, w, brow0;
         n_geometry(p, ti.jn, n_mma, w, brow0);
@@ -451,9 +456,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t tempty_mma0 = map_to_cta(tempty0, 0);
     uint32_t acc = 0, acc_phase = 0;
     bool ok = true;
-    for (long long t = pair_id; ok; t += n_pairs) {
+    int e_hint = 0;
+        for (long long t = pair_id; ok; t += n_pairs) {
       TileInfo ti;
-      if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti)) break;
+      if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti, e_hint)) break;
       int n_mma, w, brow0;
       n_geometry(p, ti.jn, n_mma, w, brow0);
       const bool have_acc = ti.kblocks > 0;
