@@ -367,6 +367,14 @@ def variant_timing(wl, device, X_host, dY_host, steps, skip, min_s=1.0):
         torch.cuda.synchronize()
         res[f"combine={combine},streams={streams}"] = {"ms_per_step": e0.elapsed_time(e1) / steps, "steps": steps,
                                                        "status_word": int(lay.t["status"].item())}
+        if combine == "fused" and streams == 1:
+            # the two passes the fused combine leaves of the gather kernels, against the method's bytes
+            bd = breakdown(lay, reps=3)
+            _, alg = hbm_bytes(wl)
+            peak = measured_peaks()["hbm_gbs"]
+            res[f"combine={combine},streams={streams}"].update({
+                "combine_ms": bd["combine"], "unpermute_grad_ms": bd["unpermute_grad"],
+                "hbm_frac_of_measured_algorithmic": {k: alg[k] / (bd[k] * 1e-3) / 1e9 / peak for k in ("combine", "unpermute_grad")}})
         del lay
         torch.cuda.empty_cache()
     return res

@@ -31,9 +31,9 @@ def _sets_from_mask(mask_u64, E):
     return [[j for j in range(E) if (int(m) >> j) & 1] for m in mask_u64]
 
 
-def _run(wl):
+def _run(wl, fused_combine=False):
     import bench
-    lay, cal = bench.build_layer(wl, "cuda:0", keep=True)
+    lay, cal = bench.build_layer(wl, "cuda:0", keep=True, fused_combine=fused_combine, side_stream=fused_combine)
     X, dY = G.hidden(wl), G.grad_out(wl)
     lay.set_input(X, dY)
     lay.train_step()
@@ -108,7 +108,8 @@ def _check_sampled_tokens(wl, lay, X, dY, L, idx, sets, rank, n_sample):
     ws = f["w"].reshape(-1)[:, None]
     assert_close_abs(_dev_rows(lay.t["w_row"], rows_dev), ws[:, 0], 1e-5, "w_row")
     assert_close_elem(_dev_rows(lay.t["H"], rows_dev), ws * f["H"][rows_ref], what="H")
-    assert_close_rms(_dev_rows(lay.t["Yp"], rows_dev), ws * f["Yp"][rows_ref], 5e-2, "Yp", out_bf16=False)
+    if "Yp" in lay.t:  # (the fused combine keeps no per-row partials)
+        assert_close_rms(_dev_rows(lay.t["Yp"], rows_dev), ws * f["Yp"][rows_ref], 5e-2, "Yp", out_bf16=False)
     assert np.array_equal(_dev_rows(lay.t["Xp"], rows_dev), X[S].astype(np.float64).repeat(K, axis=0))
     assert_close_rms(_dev_rows(lay.t["Y"], S), f["Y"], 2e-2, "Y")
     g = O.layer_bwd(X[S], Wg, W1, W3, W2, f, dY[S], shared=sh, wsg=wsg)
@@ -116,12 +117,14 @@ def _check_sampled_tokens(wl, lay, X, dY, L, idx, sets, rank, n_sample):
     dl_ref = np.take_along_axis(g["dL"], f["idx"], axis=1)
     assert_close_rms(_dev_rows(lay.t["dl"], S), dl_ref, 2e-2, "dl", out_bf16=False)
     assert np.array_equal(_dev_rows(lay.t["dYp"], rows_dev), dY[S].astype(np.float64).repeat(K, axis=0))
-    assert_close_rms(_dev_rows(lay.t["dXp"], rows_dev), g["dXp"][rows_ref], 5e-2, "dXp", out_bf16=False)
+    if "dXp" in lay.t:
+        assert_close_rms(_dev_rows(lay.t["dXp"], rows_dev), g["dXp"][rows_ref], 5e-2, "dXp", out_bf16=False)
     assert_close_rms(_dev_rows(lay.t["dX"], S), g["dX"], 2e-2, "dX")
     if wl.I_s:
         assert_close_abs(_dev_rows(lay.t["z"], S), f["z"], 1e-4, "z")
         assert_close_rms(_dev_rows(lay.t["dz"], S), g["dz"], 2e-2, "dz", out_bf16=False)
-        assert_close_rms(_dev_rows(lay.t["Ys"], S), O.sigmoid(f["z"])[:, None] * f["Ys"], 5e-2, "Ys", out_bf16=False)
+        if "Ys" in lay.t:
+            assert_close_rms(_dev_rows(lay.t["Ys"], S), O.sigmoid(f["z"])[:, None] * f["Ys"], 5e-2, "Ys", out_bf16=False)
 
 
 def _check_expert_grads(wl, lay, X, dY, w_ref, counts, offsets, sor, experts):
@@ -139,7 +142,8 @@ def _check_expert_grads(wl, lay, X, dY, w_ref, counts, offsets, sor, experts):
         A, B, H, _ = O.swiglu_fwd(Xe, cnt, off, W1[e:e + 1], W3[e:e + 1], W2[e:e + 1])
         dXp, dW1, dW3, dW2 = O.swiglu_bwd(Xe, cnt, off, W1[e:e + 1], W3[e:e + 1], W2[e:e + 1], A, B, dYpe)
         assert_close_elem(lay.t["H"][r0:r0 + n].float().cpu().numpy(), w_ref[tok, k][:, None] * H, what=f"H[{e}]")
-        assert_close_rms(lay.t["dXp"][r0:r0 + n].cpu().numpy(), dXp, 5e-2, f"dXp[{e}]", out_bf16=False)
+        if "dXp" in lay.t:
+            assert_close_rms(lay.t["dXp"][r0:r0 + n].cpu().numpy(), dXp, 5e-2, f"dXp[{e}]", out_bf16=False)
         # error scale of each gradient element: sqrt(sum over the expert's rows of (term)^2), see assert_close_contraction
         sg = O.sigmoid(A)
         dH = dYpe @ np.asarray(W2[e], np.float64)
@@ -171,10 +175,12 @@ def _check_shared_slabs(wl, lay, X, dY, slabs, width=64):
         assert_close_rms(lay.t["dWs2"][0][:, sl].float().cpu().numpy(), dW2, 2e-2, f"dWs2[:, {j0}:]")
 
 
-@pytest.mark.parametrize("name", ["c3", "c2", "c5"])
-def test_fullsize_train_step(name):
+@pytest.mark.parametrize("name,fused_combine", [("c3", False), ("c2", False), ("c5", False), ("c3", True)])
+def test_fullsize_train_step(name, fused_combine):
+    """fused_combine: the same step with the combine folded into the GEMM epilogues and the shared expert on a second
+    stream (the variant bench.py times beside its main line)."""
     wl = G.WORKLOADS[name]
-    lay, cal, X, dY = _run(wl)
+    lay, cal, X, dY = _run(wl, fused_combine)
     sets, part, rank = _check_calibration(wl, cal)
     L, idx, w_ref, counts, offsets, ros, sor = _check_integer_path(wl, lay, sets, part, rank)
     assert int(counts.sum()) == wl.N * wl.K
