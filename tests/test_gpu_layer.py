@@ -433,3 +433,62 @@ def test_fused_combine_matches_oracle(name, N, d, E, I, K, T, P, I_s, bf16):
     g = O.layer_bwd(X[S], Wg, W1, W3, W2, f2, dY[S], shared=sh, wsg=wsg)
     close(lay.host("dX")[S][same], g["dX"][same], "dX (fused combine)")
     _close(bf16, stored_bf16=False)(lay.host("dw")[S][same], g["dw"][same], "dw (fused combine)")
+
+
+def _random_shape(seed):
+    rng = np.random.default_rng(1000 + seed)
+    E = int(rng.integers(1, 13))
+    K = int(rng.integers(1, min(E, 4) + 1))
+    T = int(rng.integers(K - 1, E)) if E > 1 else 0
+    return dict(N=int(rng.integers(1, 900)), d=16 * int(rng.integers(1, 33)), E=E, I=16 * int(rng.integers(1, 26)), K=K, T=T,
+                P=int(rng.integers(1, E + 1)), I_s=int(rng.choice([0, 16 * int(rng.integers(1, 20))])) if E < 12 else 0)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_shapes_bf16_layer(seed):
+    """Randomly drawn layer shapes (token count, widths that are multiples of 16 only, expert count, K, T, with
+    and without a shared expert) through the tensor-core drivers: routing and index bit-exact, Y / dX and every
+    parameter gradient on the bars of the edge-shape test."""
+    sh_ = _random_shape(seed)
+    wl = G.Workload(f"rnd{seed}", bf16=True, seed=40 + seed, **sh_)
+    N, E, K, T, I_s = wl.N, wl.E, wl.K, wl.T, wl.I_s
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    sh = G.shared_weights(wl) if I_s else None
+    sets = random_sets(E, T, seed=seed) if T > 0 else np.zeros((E, 0), dtype=np.int64)
+    rank = np.random.default_rng(seed).permutation(E)
+    lay = _layer(wl, backward=True, side_stream=bool(seed & 1))
+    lay.set_params(Wg, W1, W3, W2, wsg, sh)
+    lay.set_routing(mask=mask_of(sets, E) if T > 0 else None, expert_rank=rank)
+    lay.set_input(X, dY)
+    lay.forward()
+    lay.backward()
+    torch.cuda.synchronize()
+    assert int(lay.t["status"].item()) == 0, sh_
+    f = O.layer_fwd(X, Wg, W1, W3, W2, sets if T > 0 else None, K, expert_rank=rank, row_align=lay.cfg.row_align, shared=sh,
+                    wsg=wsg, logits=lay.host("L"))
+    assert np.array_equal(lay.host("idx"), f["idx"]), sh_
+    assert np.array_equal(lay.host("row_of_slot"), f["row_of_slot"]) and np.array_equal(lay.host("offsets"), f["offsets"])
+    live = live_rows(f["counts"], f["offsets"])
+    assert_close_elem(lay.host("H")[live], (row_weights(f)[:, None] * f["H"])[live], what="H")
+    assert_close_rms(lay.host("Y"), f["Y"], 2e-2, "Y")
+    f2 = O.layer_fwd(X, Wg, W1, W3, W2, sets if T > 0 else None, K, expert_rank=rank, row_align=lay.cfg.row_align, shared=sh,
+                     wsg=wsg)
+    if not np.array_equal(f2["idx"], f["idx"]):
+        pytest.skip("fp32 and fp64 logits disagree on a near-tie; backward parity needs equal routing")
+    g = O.layer_bwd(X, Wg, W1, W3, W2, f2, dY, shared=sh, wsg=wsg)
+    grads = [host(t) for t in lay.unpacked_grads()]
+    few = dict(frac=6e-2 if N < 8 * E else 3e-2, ulps=4.0, rms_frac=1e-2)  # few rows per expert: see the edge-shape test
+    for e in range(E):
+        for got, ref, nm in ((grads[0][e], g["dW1"][e], "dW1"), (grads[1][e], g["dW3"][e], "dW3"),
+                             (lay.host("dW2")[e], g["dW2"][e], "dW2")):
+            if f["counts"][e] == 0:
+                assert not got.any(), f"{nm}[{e}] of an expert without tokens"
+            else:
+                assert_close_rms(got, ref, what=f"{nm}[{e}] random shape", **few)
+    assert_close_rms(lay.host("dX"), g["dX"], what="dX random shape", **few)
+    assert_close_rms(lay.host("dWg"), g["dWg"], what="dWg random shape", **few)
+    if I_s:
+        assert_close_rms(grads[2], g["dWs1"], what="dWs1 random shape", **few)
+        assert_close_rms(lay.host("dWs2")[0], g["dWs2"], what="dWs2 random shape", **few)
