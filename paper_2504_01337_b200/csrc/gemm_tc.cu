@@ -314,8 +314,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (!decode_tile(p, s_off, s_cnt, s_pt, t, ti, e_hint)) break;
           int n_mma, w, brow0;
           n_geometry(p, ti.jn, n_mma, w, brow0);
-          const int a0 = ti.m0 + BM * (int)rank;               // this CTA's A rows (or output-row range for MN-major A)
+          int a0 = ti.m0 + BM * (int)rank;                     // this CTA's A rows (or output-row range for MN-major A)
           const int b0 = brow0 + (n_mma >> 1) * (int)rank;     // this CTA's B rows
+          // The odd CTA's half of an expert's last tile may lie past the expert's segment: its rows would be another
+          // expert's, computed and thrown away.  Loading from beyond the array instead makes TMA fill zeros without
+          // touching memory: no operand traffic for that half, and a tensor core that multiplies zeros draws less power.
+          if (!A_MN && p.mode == TC_ROWS && a0 >= ti.m_end) a0 = p.R;
           for (int kb = 0; kb < ti.kblocks; ++kb) {
             if (!mbar_wait(empty0 + 8 * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
             if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * STAGE_BYTES);
