@@ -3,8 +3,8 @@
 // The product is HBM-bound (X is read once, E <= 64 output columns), so the kernel is a streaming
 // one: a CTA owns 128-token tiles, TMA brings [128 x 64] blocks of X and the matching [64 x 64]
 // block of Wg (rows >= E are zero-filled by the tensor map) and [16 x 64] block of wsg (row 0 is
-// the vector, rows 1..15 zero fill) through a 6-stage ring, one thread issues two tcgen05 MMAs per
-// 16 k-elements (N = 64 for the routed gate, N = 16 for the shared-expert gate) into tensor
+// the vector, rows 1..15 zero fill) through an 8-stage ring, one thread issues one tcgen05 MMA per
+// 16 k-elements (N = 64 for the routed gate, N = 80 when the shared-expert gate's block rides along) into tensor
 // memory, and four warps write the fp32 accumulators out.  Waits are bounded like in the grouped
 // GEMM kernel.
 #include "gemm.h"
@@ -12,7 +12,7 @@
 
 namespace c2r {
 
-constexpr int GT_STAGES = 6;
+constexpr int GT_STAGES = 8;
 constexpr int GT_X_BYTES = BM * BK * 2;    // 16 KB
 constexpr int GT_W_BYTES = 64 * BK * 2;    //  8 KB
 constexpr int GT_S_BYTES = 16 * BK * 2;    //  2 KB
@@ -77,8 +77,9 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
   } else if (warp == 1) {
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
-      const uint32_t idesc_w = instr_desc(n_mma, false, false);
-      const uint32_t idesc_s = instr_desc(16, false, false);
+      // with a shared gate, its [16 x 64] block follows the [64 x 64] block of Wg in shared memory (same 128-byte
+      // swizzle rows), so one MMA of N = 80 covers both: accumulator columns 0..63 logits, 64 the shared gate
+      const uint32_t idesc_w = instr_desc(has_shared ? 80 : n_mma, false, false);
       bool ok = true;
       for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
         if (!mbar_wait(tempty0 + 8 * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -88,13 +89,12 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
           if (!mbar_wait(full0 + 8 * stage, phase, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sx = smem_base + stage * GT_STAGE_BYTES;
-          const uint32_t sw = sx + GT_X_BYTES, ss = sw + GT_W_BYTES;
+          const uint32_t sw = sx + GT_X_BYTES;
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             const uint64_t da = smem_desc(sx + k * 32, 16, 1024);
             const uint32_t accum = (kb > 0 || k > 0) ? 1u : 0u;
             tc_mma(d_tmem, da, smem_desc(sw + k * 32, 16, 1024), idesc_w, accum);
-            if (has_shared) tc_mma(d_tmem + 64, da, smem_desc(ss + k * 32, 16, 1024), idesc_s, accum);
           }
           tc_commit(empty0 + 8 * stage);
           if (++stage == GT_STAGES) { stage = 0; phase ^= 1u; }
