@@ -279,7 +279,10 @@ int c2r_combine(const c2r_config* cfg, const void* Yp, const float* w, const int
 
 /* Backward of c2r_combine: dYp[row(t,k),:] = w[t,k] dY[t,:] (padding rows zeroed);
  * dw[t,k] = <dY[t,:], Yp[row(t,k),:]>; dYs = sigmoid(z) dY; dz = <dY,Ys> sigmoid'(z).
- * dY [N,d] T; Yp, Ys float; out: dYp [R,d] T; dYs [N,d] T; dw [N,K], dz [N] float. */
+ * dY [N,d] T; Yp, Ys float; out: dYp [R,d] T; dYs [N,d] T; dw [N,K], dz [N] float.
+ * For callers that keep the weights outside the expert calls (c2r_combine with w, z); the layer drivers apply
+ * them as the experts' row scale instead and get the same gradients from c2r_permute_rows, the backward expert
+ * call's qpart and c2r_route_bwd_scaled, without reading Yp. */
 int c2r_combine_bwd(const c2r_config* cfg, const void* dY, const void* Yp, const float* w,
                     const int32_t* row_of_slot, const int32_t* slot_of_row, const void* Ys, const float* z,
                     void* dYp, float* dw, void* dYs, float* dz, void* stream);
