@@ -492,3 +492,66 @@ def test_random_shapes_bf16_layer(seed):
     if I_s:
         assert_close_rms(grads[2], g["dWs1"], what="dWs1 random shape", **few)
         assert_close_rms(lay.host("dWs2")[0], g["dWs2"], what="dWs2 random shape", **few)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_call_by_call_with_the_weights_outside_the_expert_calls(bf16):
+    """The textbook chain, call by call through the C ABI: unscaled expert calls, c2r_combine with the weights,
+    c2r_combine_bwd (dYp = w dY, dw = <dY, Yp>), c2r_route_bwd, c2r_gate_bwd, c2r_unpermute_grad -- the form the
+    layer drivers replace by the row scale.  Every intermediate against the oracle's own (unscaled) tensors."""
+    b = B()
+    wl = G.Workload("cbc", N=700, d=128, E=6, I=144, K=3, T=4, P=2, I_s=80, bf16=bf16, seed=21)
+    N, E, K = wl.N, wl.E, wl.K
+    close, close32 = _close(bf16), _close(bf16, stored_bf16=False)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    Wg = Wg if bf16 else Wg * 8
+    W1, W3, W2 = G.expert_weights(wl)
+    sh = G.shared_weights(wl)
+    sets = random_sets(E, wl.T, seed=2)
+    lay = _layer(wl, backward=True)
+    lay.set_params(Wg, W1, W3, W2, wsg, sh)
+    lay.set_routing(mask=mask_of(sets, E))
+    lay.set_input(X, dY)
+    c, t, R = lay.cfg, lay.t, lay.R
+    t["dYs"] = torch.empty_like(t["dY"])
+    b.gate_logits(c, t["X"], t["Wg"], t["wsg"], t["L"], t["z"])
+    b.route(c, t["L"], t["mask"], t["idx"], t["w"], None, t["status"])
+    b.permute(c, t["idx"], None, t["X"], t["counts"], t["offsets"], t["row_of_slot"], t["slot_of_row"], t["Xp"], t["status"], t["ws"])
+    b.grouped_swiglu_fwd(c, E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["Yp"], t["status"])
+    b.grouped_swiglu_fwd(c, 1, c.I_s, N, t["X"], t["s_counts"], t["s_offsets"], t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["Ys"], t["status"])
+    b.combine(c, t["Yp"], t["w"], t["row_of_slot"], t["Ys"], t["z"], t["Y"])
+    b.combine_bwd(c, t["dY"], t["Yp"], t["w"], t["row_of_slot"], t["slot_of_row"], t["Ys"], t["z"], t["dYp"], t["dw"], t["dYs"], t["dz"])
+    b.grouped_swiglu_bwd(c, E, c.I, R, t["Xp"], t["counts"], t["offsets"], t["W13p"], t["W2"], t["AB"], t["H"], t["dYp"], t["dAB"],
+                         t["dXp"], t["dW13p"], t["dW2"], False, t["status"])
+    b.grouped_swiglu_bwd(c, 1, c.I_s, N, t["X"], t["s_counts"], t["s_offsets"], t["Ws13p"], t["Ws2"], t["ABs"], t["Hs"], t["dYs"],
+                         t["dABs"], t["dXs"], t["dWs13p"], t["dWs2"], False, t["status"])
+    b.route_bwd(c, t["w"], t["dw"], t["dl"])
+    b.gate_bwd(c, t["X"], t["Xp"], t["counts"], t["offsets"], t["slot_of_row"], t["dl"], t["dz"], t["dWg"], t["dwsg"], t["ws"])
+    b.unpermute_grad(c, t["dXp"], t["row_of_slot"], t["dXs"], t["idx"], t["dl"], t["Wg"], t["dz"], t["wsg"], t["dX"])
+    torch.cuda.synchronize()
+    assert int(t["status"].item()) == 0
+    f = O.layer_fwd(X, Wg, W1, W3, W2, sets, K, row_align=c.row_align, shared=sh, wsg=wsg, logits=lay.host("L"))
+    assert np.array_equal(lay.host("idx"), f["idx"]) and np.array_equal(lay.host("row_of_slot"), f["row_of_slot"])
+    live = live_rows(f["counts"], f["offsets"])
+    mid = (lambda g_, r_, what: assert_close_elem(g_, r_, what=what)) if bf16 else close
+    part = (lambda g_, r_, what: assert_close_rms(g_, r_, 5e-2, what, out_bf16=False)) if bf16 else close
+    mid(lay.host("H")[live], f["H"][live], "H (unscaled)")
+    part(lay.host("Yp")[live], f["Yp"][live], "Yp (unscaled)")
+    part(lay.host("Ys"), f["Ys"], "Ys (ungated)")
+    close(lay.host("Y"), f["Y"], "Y (weights in the combine)")
+    f2 = O.layer_fwd(X, Wg, W1, W3, W2, sets, K, row_align=c.row_align, shared=sh, wsg=wsg)
+    if not np.array_equal(f2["idx"], f["idx"]):
+        pytest.skip("fp32 and fp64 logits disagree on a near-tie; backward parity needs equal routing")
+    g = O.layer_bwd(X, Wg, W1, W3, W2, f2, dY, shared=sh, wsg=wsg)
+    mid(lay.host("dYp")[live], g["dYp"][live], "dYp = w dY")
+    mid(host(t["dYs"]), g["dYs"], "dYs = sigmoid(z) dY")
+    close32(lay.host("dw"), g["dw"], "dw = <dY, Yp>")
+    close32(lay.host("dz"), g["dz"], "dz")
+    close32(lay.host("dl"), np.take_along_axis(g["dL"], f["idx"], axis=1), "dl")
+    part(lay.host("dXp")[live], g["dXp"][live], "dXp")
+    grads = [host(x) for x in lay.unpacked_grads()]
+    close(grads[0], g["dW1"], "dW1"); close(grads[1], g["dW3"], "dW3"); close(lay.host("dW2"), g["dW2"], "dW2")
+    close(grads[2], g["dWs1"], "dWs1"); close(lay.host("dWs2")[0], g["dWs2"], "dWs2")
+    close32(lay.host("dWg"), g["dWg"], "dWg"); close32(lay.host("dwsg"), g["dwsg"], "dwsg")
+    close(lay.host("dX"), g["dX"], "dX")
