@@ -229,7 +229,7 @@ def breakdown(lay, reps=3):
         ("route_bwd", lambda: B.route_bwd_scaled(c, t["w"], t["row_of_slot"], qpart, nq, t.get("z"), qspart, nqs,
                                                  t["dw"], t["dl"], t.get("dz"))),
         ("gate_bwd", lambda: B.gate_bwd(c, t["X"], t.get("Xp"), t["counts"], t["offsets"], t["slot_of_row"], t["dl"],
-                                        t.get("dz"), t["dWg"], t.get("dwsg"), ws)),
+                                        t.get("dz"), t["dWg"], t.get("dwsg"), ws, idx=t["idx"])),
         ("unpermute_grad", lambda: B.unpermute_grad(c, t.get("dXp"), t["row_of_slot"],
                                                     t["dXacc"] if fcomb else t.get("dXs"), t["idx"], t["dl"],
                                                     t["Wg"], t.get("dz"), t.get("wsg"), t["dX"])),

@@ -307,10 +307,11 @@ int c2r_route_bwd_scaled(const c2r_config* cfg, const float* w, const int32_t* r
  * ws: C2R_WS_GATE_BWD bytes.
  * bf16 with X and ws given: evaluated as one tensor-core GEMM dL^T X over a dense [N,64] bf16 copy of the
  * gradient w.r.t. the logits (dl and dz rounded to bf16, fp32 accumulation, token splits added in a fixed
- * order); otherwise a row-serial fp32 kernel over Xp. */
+ * order); otherwise a row-serial fp32 kernel over Xp.  idx [N,K] (optional): with it the dense copy is written
+ * token by token in one pass; without it, it is zeroed and filled expert by expert through slot_of_row. */
 int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
-                 const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
-                 float* dWg, float* dwsg, int accumulate, void* ws, size_t ws_bytes, void* stream);
+                 const int32_t* offsets, const int32_t* slot_of_row, const int32_t* idx, const float* dl,
+                 const float* dz, float* dWg, float* dwsg, int accumulate, void* ws, size_t ws_bytes, void* stream);
 
 /* Gradient w.r.t. the hidden states (transpose of the dispatch, done as an atomic-free gather-sum):
  * dX[t,:] = sum_k dXp[row_of_slot[t*K+k],:]  + dXs[t,:]                (shared expert, optional)

@@ -93,7 +93,7 @@ _SIGS = {
     "c2r_combine": [_CFG] + [_P] * 7,
     "c2r_combine_bwd": [_CFG] + [_P] * 12,
     "c2r_route_bwd": [_CFG] + [_P] * 4,
-    "c2r_gate_bwd": [_CFG] + [_P] * 9 + [C.c_int, _P, C.c_size_t, _P],
+    "c2r_gate_bwd": [_CFG] + [_P] * 10 + [C.c_int, _P, C.c_size_t, _P],
     "c2r_unpermute_grad": [_CFG] + [_P] * 9 + [C.c_int, _P],
     "c2r_dispatch_volume": [_CFG] + [_P] * 6,
     "c2r_layer_fwd": [_CFG, C.POINTER(LayerBuffers), _P],
@@ -258,8 +258,8 @@ def route_bwd(cfg, w, dw, dl):
     _call("c2r_route_bwd", C.byref(cfg), _ptr(w), _ptr(dw), _ptr(dl), _stream())
 
 
-def gate_bwd(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws, accumulate=False):
-    _call("c2r_gate_bwd", C.byref(cfg), _ptr(X), _ptr(Xp), _ptr(counts), _ptr(offsets), _ptr(slot_of_row), _ptr(dl),
+def gate_bwd(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, ws, accumulate=False, idx=None):
+    _call("c2r_gate_bwd", C.byref(cfg), _ptr(X), _ptr(Xp), _ptr(counts), _ptr(offsets), _ptr(slot_of_row), _ptr(idx), _ptr(dl),
           _ptr(dz), _ptr(dWg), _ptr(dwsg), int(accumulate), _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
           _stream())
 

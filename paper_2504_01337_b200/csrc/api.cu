@@ -299,7 +299,7 @@ extern "C" int c2r_layer_bwd(const c2r_config* cfg, const c2r_layer_buffers* b, 
   if (!fcomb) C2R_TRY(ss.join());
   C2R_TRY(c2r_route_bwd_scaled(cfg, b->w, b->row_of_slot, ws.qpart, ws.nq, shared ? b->z : nullptr, ws.qspart, ws.nqs, b->dw,
                                b->dl, shared ? b->dz : nullptr, stream));
-  C2R_TRY(c2r_gate_bwd(cfg, b->X, b->Xp, b->counts, b->offsets, b->slot_of_row, b->dl, shared ? b->dz : nullptr,
+  C2R_TRY(c2r_gate_bwd(cfg, b->X, b->Xp, b->counts, b->offsets, b->slot_of_row, b->idx, b->dl, shared ? b->dz : nullptr,
                        b->dWg, shared ? b->dwsg : nullptr, accumulate, ws.gate_bwd, align256(gate_bwd_ws_bytes(cfg)),
                        stream));
   C2R_TRY(c2r_unpermute_grad(cfg, fcomb ? nullptr : b->dXp, b->row_of_slot,

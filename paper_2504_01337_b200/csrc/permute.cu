@@ -622,6 +622,31 @@ __global__ void __launch_bounds__(256) gate_dl_scatter_kernel(const int32_t* __r
     if (sl >= 0) dLd[(size_t)(sl / K) * GW_COLS + e] = __float2bfloat16_rn(dl[sl]);
   }
 }
+// The whole dense row of a token in one pass (needs idx): a warp per token, lane l owns columns 2l and 2l+1, so
+// the row leaves as one 128-byte store and neither a memset nor the per-expert scatter is needed.  Block 0 also
+// writes the split table.
+__global__ void __launch_bounds__(256) gate_dl_dense_kernel(const int32_t* __restrict__ idx, const float* __restrict__ dl,
+                                                            const float* __restrict__ dz, __nv_bfloat16* __restrict__ dLd,
+                                                            int N, int E, int K, int per, int splits,
+                                                            int32_t* __restrict__ split_counts,
+                                                            int32_t* __restrict__ split_offsets) {
+  if (blockIdx.x == 0 && (int)threadIdx.x <= splits) {
+    const int lo = min(N, (int)threadIdx.x * per);
+    split_offsets[threadIdx.x] = lo;
+    if ((int)threadIdx.x < splits) split_counts[threadIdx.x] = min(N, lo + per) - lo;
+  }
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= N) return;  // warp-uniform
+  float v0 = 0.f, v1 = 0.f;
+  for (int k = 0; k < K; ++k) {
+    const int e = min(max(idx[(size_t)t * K + k], 0), E - 1);
+    const float g = dl[(size_t)t * K + k];
+    if ((e >> 1) == lane) { if (e & 1) v1 = g; else v0 = g; }
+  }
+  if (dz != nullptr && (E >> 1) == lane) { if (E & 1) v1 = dz[t]; else v0 = dz[t]; }
+  reinterpret_cast<__nv_bfloat162*>(dLd + (size_t)t * GW_COLS)[lane] = __floats2bfloat162_rn(v0, v1);
+}
 // shared-gate column and the split table
 __global__ void __launch_bounds__(256) gate_dz_kernel(const float* __restrict__ dz, __nv_bfloat16* __restrict__ dLd, int N,
                                                       int E, int per, int splits, int32_t* __restrict__ split_counts,
@@ -819,8 +844,8 @@ extern "C" int c2r_combine_bwd(const c2r_config* cfg, const void* dY, const void
 
 template <typename T>
 static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
-                           const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
-                           float* dWg, float* dwsg, int accumulate, void* ws, cudaStream_t s) {
+                           const int32_t* offsets, const int32_t* slot_of_row, const int32_t* idx, const float* dl,
+                           const float* dz, float* dWg, float* dwsg, int accumulate, void* ws, cudaStream_t s) {
   using V = Vec16<T>;
   if (sizeof(T) == 2 && X != nullptr && ws != nullptr && cfg->N > 0 && cfg->d % 16 == 0 && cfg->E < GW_COLS &&
       ((uintptr_t)X & 15u) == 0 && tc_supported(cfg, 1, 16, cfg->N)) {
@@ -829,11 +854,16 @@ static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp,
     float* partial = (float*)((char*)ws + g.off_partial);
     int32_t* sc = (int32_t*)((char*)ws + g.off_counts);
     int32_t* so = sc + g.splits;
-    C2R_CUDA(cudaMemsetAsync(dLd, 0, (size_t)cfg->N * GW_COLS * 2, s));
-    gate_dl_scatter_kernel<<<cfg->E, 256, 0, s>>>(counts, offsets, slot_of_row, dl, dLd, cfg->K);
-    C2R_LAUNCH_CHECK();
-    gate_dz_kernel<<<(cfg->N + 255) / 256, 256, 0, s>>>(dz, dLd, cfg->N, cfg->E, g.per, g.splits, sc, so);
-    C2R_LAUNCH_CHECK();
+    if (idx != nullptr) {
+      gate_dl_dense_kernel<<<(cfg->N + 7) / 8, 256, 0, s>>>(idx, dl, dz, dLd, cfg->N, cfg->E, cfg->K, g.per, g.splits, sc, so);
+      C2R_LAUNCH_CHECK();
+    } else {
+      C2R_CUDA(cudaMemsetAsync(dLd, 0, (size_t)cfg->N * GW_COLS * 2, s));
+      gate_dl_scatter_kernel<<<cfg->E, 256, 0, s>>>(counts, offsets, slot_of_row, dl, dLd, cfg->K);
+      C2R_LAUNCH_CHECK();
+      gate_dz_kernel<<<(cfg->N + 255) / 256, 256, 0, s>>>(dz, dLd, cfg->N, cfg->E, g.per, g.splits, sc, so);
+      C2R_LAUNCH_CHECK();
+    }
     int rc = tc_gate_wgrad(cfg, X, dLd, partial, g.splits, sc, so, nullptr, s);
     if (rc) return rc;
     gate_wgrad_reduce_kernel<<<dim3((cfg->d + 255) / 256, cfg->E + 1), 256, 0, s>>>(partial, g.splits, cfg->E, cfg->d,
@@ -856,8 +886,9 @@ static int gate_bwd_launch(const c2r_config* cfg, const void* X, const void* Xp,
 }
 
 extern "C" int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp, const int32_t* counts,
-                            const int32_t* offsets, const int32_t* slot_of_row, const float* dl, const float* dz,
-                            float* dWg, float* dwsg, int accumulate, void* ws, size_t ws_bytes, void* stream) {
+                            const int32_t* offsets, const int32_t* slot_of_row, const int32_t* idx, const float* dl,
+                            const float* dz, float* dWg, float* dwsg, int accumulate, void* ws, size_t ws_bytes,
+                            void* stream) {
   int rc = check_config(cfg);
   if (rc) return rc;
   C2R_REQUIRE(counts && offsets && slot_of_row && dl && dWg, C2R_ERR_INVALID_ARG);
@@ -865,9 +896,9 @@ extern "C" int c2r_gate_bwd(const c2r_config* cfg, const void* X, const void* Xp
   C2R_REQUIRE(!dz || (ws && ws_bytes >= gate_bwd_ws_bytes(cfg)), C2R_ERR_WORKSPACE);
   if (ws && ws_bytes < gate_bwd_ws_bytes(cfg)) ws = nullptr;  // too small for the tensor-core form: row-serial kernel
   if (cfg->dtype == C2R_BF16)
-    return gate_bwd_launch<__nv_bfloat16>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, accumulate, ws,
+    return gate_bwd_launch<__nv_bfloat16>(cfg, X, Xp, counts, offsets, slot_of_row, idx, dl, dz, dWg, dwsg, accumulate, ws,
                                           as_stream(stream));
-  return gate_bwd_launch<float>(cfg, X, Xp, counts, offsets, slot_of_row, dl, dz, dWg, dwsg, accumulate, ws,
+  return gate_bwd_launch<float>(cfg, X, Xp, counts, offsets, slot_of_row, idx, dl, dz, dWg, dwsg, accumulate, ws,
                                 as_stream(stream));
 }
 

@@ -481,9 +481,13 @@ extern "C" int c2r_dispatch_volume(const c2r_config* cfg, const int32_t* idx, co
   const int P = cfg->P;
   C2R_REQUIRE(P >= 1 && P <= cfg->E, C2R_ERR_INVALID_ARG);
   cudaStream_t s = as_stream(stream);
-  C2R_CUDA(cudaMemsetAsync(totals, 0, 4 * sizeof(uint64_t), s));
-  C2R_CUDA(cudaMemsetAsync(send_naive, 0, sizeof(uint64_t) * P * P, s));
-  C2R_CUDA(cudaMemsetAsync(send_dedup, 0, sizeof(uint64_t) * P * P, s));
+  if (send_naive == totals + 4 && send_dedup == send_naive + P * P) {  // one buffer (the layer drivers' layout)
+    C2R_CUDA(cudaMemsetAsync(totals, 0, sizeof(uint64_t) * (4 + 2 * P * P), s));
+  } else {
+    C2R_CUDA(cudaMemsetAsync(totals, 0, 4 * sizeof(uint64_t), s));
+    C2R_CUDA(cudaMemsetAsync(send_naive, 0, sizeof(uint64_t) * P * P, s));
+    C2R_CUDA(cudaMemsetAsync(send_dedup, 0, sizeof(uint64_t) * P * P, s));
+  }
   if (cfg->N == 0) return C2R_OK;
   int blocks = (cfg->N + 255) / 256;
   if (blocks > 296) blocks = 296;
