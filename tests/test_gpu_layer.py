@@ -555,3 +555,33 @@ def test_call_by_call_with_the_weights_outside_the_expert_calls(bf16):
     close(grads[2], g["dWs1"], "dWs1"); close(lay.host("dWs2")[0], g["dWs2"], "dWs2")
     close32(lay.host("dWg"), g["dWg"], "dWg"); close32(lay.host("dwsg"), g["dwsg"], "dwsg")
     close(lay.host("dX"), g["dX"], "dX")
+
+
+@pytest.mark.parametrize("side_stream", [False, True])
+def test_train_step_replays_from_a_cuda_graph(side_stream):
+    """Nothing in the library allocates or synchronises and tensor maps travel as kernel parameters, so a training
+    step captured into a CUDA graph (after one eager step has done the per-device set-up) replays bit-identically,
+    also with the shared expert forked onto the second stream."""
+    wl = G.Workload("graph", N=2500, d=256, E=8, I=272, K=2, T=4, P=2, I_s=400, bf16=True, seed=29)
+    X = G.hidden(wl); dY = G.grad_out(wl)
+    Wg, wsg = G.gate_weights(wl)
+    W1, W3, W2 = G.expert_weights(wl)
+    lay = _layer(wl, backward=True, profile=True, side_stream=side_stream)
+    lay.set_params(Wg, W1, W3, W2, wsg, G.shared_weights(wl))
+    lay.set_routing(mask=mask_of(random_sets(wl.E, wl.T, seed=3), wl.E))
+    lay.set_input(X, dY)
+    lay.train_step()                      # eager: per-device set-up happens here, outside any capture
+    torch.cuda.synchronize()
+    names = ("Y", "dX", "dW13p", "dW2", "dWs13p", "dWs2", "dWg", "dwsg", "C", "mask_next", "idx")
+    eager = {n: lay.t[n].clone() for n in names}
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        lay.train_step()
+    for n in names:
+        lay.t[n].zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert int(lay.t["status"].item()) == 0
+    for n in names:
+        assert torch.equal(lay.t[n], eager[n]), n
