@@ -377,6 +377,28 @@ def variant_timing(wl, device, X_host, dY_host, steps, skip, min_s=1.0):
                 "hbm_frac_of_measured_algorithmic": {k: alg[k] / (bd[k] * 1e-3) / 1e9 / peak for k in ("combine", "unpermute_grad")}})
         del lay
         torch.cuda.empty_cache()
+    # the default configuration replayed from a CUDA graph (launch gaps between the 26 launches of a step removed)
+    lay = build_layer(wl, device)
+    lay.set_input(X_host.to(device), dY_host.to(device))
+    warm_up(lay, 3, 0.0)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        lay.train_step()
+    t0 = time.perf_counter()
+    while time.perf_counter() - t0 < min_s:
+        for _ in range(10):
+            graph.replay()
+        torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    res["cuda_graph_replay"] = {"ms_per_step": e0.elapsed_time(e1) / steps, "steps": steps,
+                                "status_word": int(lay.t["status"].item())}
+    del graph, lay
+    torch.cuda.empty_cache()
     return res
 
 
