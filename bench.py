@@ -711,8 +711,9 @@ def main():
                                                      cal["C"].cpu(), wl.E, wl.K, wl.T)
             out["skew_report_c4"] = skew_report(G.WORKLOADS["c4"], device)
             out["dedup_dispatch"] = dedup_dispatch_timing(lay)
-            out["variants"] = variant_timing(wl, device, X_host, dY_host, steps=max(3, min(args.steps, 20)),
-                                             skip=(args.combine, args.streams), min_s=args.min_warmup_s)
+            if world == 1:  # (a multi-rank run holds every GPU while rank 0 would time these alone)
+                out["variants"] = variant_timing(wl, device, X_host, dY_host, steps=max(3, min(args.steps, 20)),
+                                                 skip=(args.combine, args.streams), min_s=args.min_warmup_s)
         if not args.no_cpu_baseline and world == 1:
             n_tok = args.cpu_baseline_tokens
             _, st = cpu_oracle_step(wl, n_tok)      # builds the inputs (and warms the BLAS threads)
